@@ -1,0 +1,360 @@
+// Host side of the C ABI declared in dcasgd.h: argument validation, the serial message loop of
+// Algorithm 2, and the launches.  Every check runs before the first launch of a call.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "dcasgd.h"
+#include "kernels.cuh"
+#include "window_compiler.h"
+
+using namespace dcasgd;
+
+struct dcasgd_server {
+    dcasgd_config cfg;
+    Hyper h;
+    cudaStream_t stream;
+    int device;
+    uint64_t t;          // pushes applied (Algorithm 2's t)
+    uint64_t launches;   // kernels launched through this handle
+};
+
+namespace {
+
+struct Range { const char* lo; const char* hi; const char* name; };
+
+inline Range range_of(const void* p, uint64_t bytes, const char* name) {
+    return Range{static_cast<const char*>(p), static_cast<const char*>(p) + bytes, name};
+}
+inline bool overlap(const Range& a, const Range& b) {
+    return a.lo < b.hi && b.lo < a.hi && a.lo != a.hi && b.lo != b.hi;
+}
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline uint64_t grad_elem_bytes(const dcasgd_config& c) { return c.grad_dtype == DCASGD_BF16 ? 2 : 4; }
+
+int fail(int status, const char* fmt, ...) __attribute__((format(printf, 2, 3)));
+int fail(int status, const char* fmt, ...) {
+    char buf[400];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    set_error("%s", buf);
+    return status;
+}
+
+int cuda_fail(const char* what, cudaError_t e) {
+    return fail(DCASGD_ECUDA, "%s: %s (%s)", what, cudaGetErrorName(e), cudaGetErrorString(e));
+}
+
+// The state arrays of a server as byte ranges, for overlap checks against caller buffers.
+int state_ranges(const dcasgd_config& c, Range out[3]) {
+    int k = 0;
+    out[k++] = range_of(c.w, c.n * 4, "w");
+    const uint64_t bak = c.n == 0 ? 0 : ((uint64_t)(c.num_workers - 1) * c.w_bak_stride + c.n) * 4;
+    out[k++] = range_of(c.w_bak, bak, "w_bak");
+    if (c.ms) out[k++] = range_of(c.ms, c.n * 4, "ms");
+    return k;
+}
+
+int check_foreign(const dcasgd_config& c, const void* p, uint64_t bytes, const char* name) {
+    Range st[3];
+    const int k = state_ranges(c, st);
+    const Range r = range_of(p, bytes, name);
+    for (int i = 0; i < k; ++i)
+        if (overlap(r, st[i])) return fail(DCASGD_EINVAL, "%s overlaps the server's %s", name, st[i].name);
+    return DCASGD_OK;
+}
+
+inline unsigned blocks_for(uint64_t n, int vecs_per_thread) {
+    const uint64_t nvec = (n + 3) / 4;
+    const uint64_t per_block = (uint64_t)kThreads * vecs_per_thread;
+    return (unsigned)((nvec + per_block - 1) / per_block);
+}
+
+int after_launch(dcasgd_server* s, const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(what, e);
+    s->launches += 1;
+    return DCASGD_OK;
+}
+
+int launch_pull(dcasgd_server* s, uint32_t m, float* out_w) {
+    const dcasgd_config& c = s->cfg;
+    if (c.n == 0) return DCASGD_OK;
+    k_pull<<<blocks_for(c.n, kPushUnroll), kThreads, 0, s->stream>>>(
+        c.w, c.w_bak + (uint64_t)m * c.w_bak_stride, out_w, c.n);
+    return after_launch(s, "pull kernel");
+}
+
+int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
+    const dcasgd_config& c = s->cfg;
+    s->t += 1;
+    if (c.n == 0) return DCASGD_OK;
+    PushArgs a;
+    a.w = c.w;
+    a.wb_m = c.w_bak + (uint64_t)m * c.w_bak_stride;
+    a.ms = c.ms;
+    a.g = g;
+    a.n = c.n;
+    a.eta = eta < 0.0f ? c.eta : eta;
+    a.h = s->h;
+    const unsigned grid = blocks_for(c.n, kPushUnroll);
+    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
+    if (ad && bf)       k_push<true, true><<<grid, kThreads, 0, s->stream>>>(a);
+    else if (ad)        k_push<true, false><<<grid, kThreads, 0, s->stream>>>(a);
+    else if (bf)        k_push<false, true><<<grid, kThreads, 0, s->stream>>>(a);
+    else                k_push<false, false><<<grid, kThreads, 0, s->stream>>>(a);
+    return after_launch(s, "push kernel");
+}
+
+int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void* grad_pool,
+                  uint64_t grad_stride_bytes) {
+    const dcasgd_config& c = s->cfg;
+    s->t += wp.n_pushes;
+    if (c.n == 0) return DCASGD_OK;
+    if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
+    DevProgram p;
+    std::memset(&p, 0, sizeof p);
+    p.n_pushes = wp.n_pushes;
+    p.n_slots = wp.n_slots;
+    for (uint32_t j = 0; j < wp.n_pushes; ++j) {
+        p.grad_id[j] = wp.grad_id[j];
+        p.eta[j] = wp.eta[j];
+        p.src[j] = wp.src[j];
+    }
+    for (uint32_t j = 0; j <= wp.n_pushes; ++j) p.save_slot[j] = (int8_t)wp.save_slot[j];
+    for (uint32_t j = 0; j <= wp.n_pushes + 1; ++j) p.store_begin[j] = (uint8_t)wp.store_begin[j];
+    for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_worker[k] = (uint16_t)wp.store_worker[k];
+    ReplayArgs a;
+    a.w = c.w;
+    a.w_bak = c.w_bak;
+    a.ms = c.ms;
+    a.grad_pool = static_cast<const char*>(grad_pool);
+    a.stride = c.w_bak_stride;
+    a.grad_stride_bytes = grad_stride_bytes;
+    a.n = c.n;
+    a.h = s->h;
+    const unsigned grid = blocks_for(c.n, 1);
+    const size_t smem = (size_t)wp.n_slots * kThreads * sizeof(float4);
+    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
+    if (ad && bf)       k_replay<true, true><<<grid, kThreads, smem, s->stream>>>(a, p);
+    else if (ad)        k_replay<true, false><<<grid, kThreads, smem, s->stream>>>(a, p);
+    else if (bf)        k_replay<false, true><<<grid, kThreads, smem, s->stream>>>(a, p);
+    else                k_replay<false, false><<<grid, kThreads, smem, s->stream>>>(a, p);
+    return after_launch(s, "window replay kernel");
+}
+
+template <class K>
+cudaError_t allow_slots(K kernel) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                DCASGD_MAX_WINDOW_SLOTS * kThreads * (int)sizeof(float4));
+}
+
+int check_server(const dcasgd_server* s, const char* fn) {
+    if (!s) return fail(DCASGD_EINVAL, "%s: server is NULL", fn);
+    int dev = -1;
+    const cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(fn, e);
+    if (dev != s->device) return fail(DCASGD_EINVAL, "%s: current device %d is not the server's device %d", fn, dev, s->device);
+    return DCASGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* dcasgd_last_error(void) { return get_error(); }
+
+const char* dcasgd_status_string(int status) {
+    switch (status) {
+        case DCASGD_OK: return "DCASGD_OK";
+        case DCASGD_EINVAL: return "DCASGD_EINVAL";
+        case DCASGD_EWORKER: return "DCASGD_EWORKER";
+        case DCASGD_EALIGN: return "DCASGD_EALIGN";
+        case DCASGD_ELOG: return "DCASGD_ELOG";
+        case DCASGD_ECUDA: return "DCASGD_ECUDA";
+        case DCASGD_ENOMEM: return "DCASGD_ENOMEM";
+        default: return "DCASGD_<unknown>";
+    }
+}
+
+uint32_t dcasgd_version(void) { return DCASGD_VERSION; }
+
+int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
+    if (!cfg || !out) return fail(DCASGD_EINVAL, "dcasgd_create: NULL argument");
+    *out = nullptr;
+    const dcasgd_config& c = *cfg;
+    if (c.num_workers == 0 || c.num_workers > 65535u)
+        return fail(DCASGD_EINVAL, "dcasgd_create: num_workers must be 1..65535 (got %u)", c.num_workers);
+    if (c.variant > DCASGD_ADAPTIVE) return fail(DCASGD_EINVAL, "dcasgd_create: unknown variant %u", c.variant);
+    if (c.grad_dtype > DCASGD_BF16) return fail(DCASGD_EINVAL, "dcasgd_create: unknown grad_dtype %u", c.grad_dtype);
+    if (!std::isfinite(c.eta) || c.eta < 0.0f) return fail(DCASGD_EINVAL, "dcasgd_create: eta must be finite and >= 0");
+    if (!std::isfinite(c.lambda)) return fail(DCASGD_EINVAL, "dcasgd_create: lambda must be finite");
+    const bool adaptive = c.variant == DCASGD_ADAPTIVE;
+    if (adaptive) {
+        if (!(c.mu >= 0.0f && c.mu < 1.0f)) return fail(DCASGD_EINVAL, "dcasgd_create: mu must be in [0,1)");
+        if (!(std::isfinite(c.eps) && c.eps >= 0.0f)) return fail(DCASGD_EINVAL, "dcasgd_create: eps must be finite and >= 0");
+        if (!c.ms && c.n) return fail(DCASGD_EINVAL, "dcasgd_create: the adaptive variant needs ms");
+    } else if (c.ms) {
+        return fail(DCASGD_EINVAL, "dcasgd_create: ms must be NULL for the constant variant");
+    }
+    if (c.n) {
+        if (!c.w || !c.w_bak) return fail(DCASGD_EINVAL, "dcasgd_create: w and w_bak are required");
+        if (c.w_bak_stride < c.n) return fail(DCASGD_EINVAL, "dcasgd_create: w_bak_stride < n");
+        if (c.w_bak_stride % 4) return fail(DCASGD_EALIGN, "dcasgd_create: w_bak_stride must be a multiple of 4 floats");
+        if (!aligned16(c.w) || !aligned16(c.w_bak) || (c.ms && !aligned16(c.ms)))
+            return fail(DCASGD_EALIGN, "dcasgd_create: w, w_bak and ms must be 16-byte aligned");
+        if (c.n > (uint64_t)1 << 40) return fail(DCASGD_EINVAL, "dcasgd_create: n too large");
+        Range st[3];
+        const int k = state_ranges(c, st);
+        for (int i = 0; i < k; ++i)
+            for (int j = i + 1; j < k; ++j)
+                if (overlap(st[i], st[j]))
+                    return fail(DCASGD_EINVAL, "dcasgd_create: %s overlaps %s", st[i].name, st[j].name);
+    }
+
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("dcasgd_create: cudaGetDevice", e);
+    if (c.n) {
+        const void* ptrs[3] = {c.w, c.w_bak, c.ms};
+        const char* names[3] = {"w", "w_bak", "ms"};
+        for (int i = 0; i < 3; ++i) {
+            if (!ptrs[i]) continue;
+            cudaPointerAttributes at;
+            e = cudaPointerGetAttributes(&at, ptrs[i]);
+            if (e != cudaSuccess) return cuda_fail("dcasgd_create: cudaPointerGetAttributes", e);
+            if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged)
+                return fail(DCASGD_EINVAL, "dcasgd_create: %s is not device memory", names[i]);
+            if (at.type == cudaMemoryTypeDevice && at.device != dev)
+                return fail(DCASGD_EINVAL, "dcasgd_create: %s lives on device %d, current device is %d", names[i], at.device, dev);
+        }
+    }
+    if ((e = allow_slots(k_replay<false, false>)) != cudaSuccess || (e = allow_slots(k_replay<false, true>)) != cudaSuccess ||
+        (e = allow_slots(k_replay<true, false>)) != cudaSuccess || (e = allow_slots(k_replay<true, true>)) != cudaSuccess)
+        return cuda_fail("dcasgd_create: cudaFuncSetAttribute", e);
+
+    dcasgd_server* s = new (std::nothrow) dcasgd_server;
+    if (!s) return fail(DCASGD_ENOMEM, "dcasgd_create: out of host memory");
+    s->cfg = c;
+    s->h.lambda = c.lambda;
+    s->h.mu = adaptive ? c.mu : 0.0f;
+    s->h.omm = 1.0f - s->h.mu;
+    s->h.eps = adaptive ? c.eps : 0.0f;
+    s->stream = static_cast<cudaStream_t>(c.stream);
+    s->device = dev;
+    s->t = 0;
+    s->launches = 0;
+    if (c.n) {
+        // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
+        k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
+        const int rc = after_launch(s, "init kernel");
+        if (rc != DCASGD_OK) { delete s; return rc; }
+    }
+    *out = s;
+    return DCASGD_OK;
+}
+
+int dcasgd_pull(dcasgd_server* s, uint32_t m, float* out_w) {
+    int rc = check_server(s, "dcasgd_pull");
+    if (rc) return rc;
+    if (m >= s->cfg.num_workers) return fail(DCASGD_EWORKER, "dcasgd_pull: worker %u >= %u", m, s->cfg.num_workers);
+    if (out_w && s->cfg.n) {
+        if (!aligned16(out_w)) return fail(DCASGD_EALIGN, "dcasgd_pull: out_w must be 16-byte aligned");
+        if ((rc = check_foreign(s->cfg, out_w, s->cfg.n * 4, "out_w"))) return rc;
+    }
+    return launch_pull(s, m, out_w);
+}
+
+int dcasgd_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
+    int rc = check_server(s, "dcasgd_push");
+    if (rc) return rc;
+    if (m >= s->cfg.num_workers) return fail(DCASGD_EWORKER, "dcasgd_push: worker %u >= %u", m, s->cfg.num_workers);
+    if (!std::isfinite(eta)) return fail(DCASGD_EINVAL, "dcasgd_push: eta is not finite");
+    if (s->cfg.n) {
+        if (!g) return fail(DCASGD_EINVAL, "dcasgd_push: g is NULL");
+        if (!aligned16(g)) return fail(DCASGD_EALIGN, "dcasgd_push: g must be 16-byte aligned");
+        if ((rc = check_foreign(s->cfg, g, s->cfg.n * grad_elem_bytes(s->cfg), "g"))) return rc;
+    }
+    return launch_push(s, m, g, eta);
+}
+
+int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, const void* grad_pool,
+                     uint64_t grad_stride_bytes, uint32_t num_grads, uint32_t window_k) {
+    int rc = check_server(s, "dcasgd_apply_log");
+    if (rc) return rc;
+    const dcasgd_config& c = s->cfg;
+    if (window_k == 0) return fail(DCASGD_EINVAL, "dcasgd_apply_log: window_k must be >= 1");
+    if (count == 0) return DCASGD_OK;
+    if (!ev) return fail(DCASGD_EINVAL, "dcasgd_apply_log: ev is NULL");
+    // the whole log is checked before anything is launched
+    bool any_push = false;
+    for (uint64_t r = 0; r < count; ++r) {
+        if (ev[r].kind > DCASGD_PUSH) return fail(DCASGD_ELOG, "log record %llu: unknown kind %u", (unsigned long long)r, ev[r].kind);
+        if (ev[r].worker >= c.num_workers) return fail(DCASGD_ELOG, "log record %llu: worker %u >= %u", (unsigned long long)r, ev[r].worker, c.num_workers);
+        if (ev[r].kind == DCASGD_PUSH) {
+            any_push = true;
+            if (ev[r].grad_id >= num_grads) return fail(DCASGD_ELOG, "log record %llu: grad_id %u >= %u", (unsigned long long)r, ev[r].grad_id, num_grads);
+            if (!std::isfinite(ev[r].eta)) return fail(DCASGD_ELOG, "log record %llu: eta is not finite", (unsigned long long)r);
+        }
+    }
+    const uint64_t gbytes = c.n * grad_elem_bytes(c);
+    if (any_push && c.n) {
+        if (!grad_pool) return fail(DCASGD_EINVAL, "dcasgd_apply_log: grad_pool is NULL");
+        if (!aligned16(grad_pool) || grad_stride_bytes % 16) return fail(DCASGD_EALIGN, "dcasgd_apply_log: grad_pool and grad_stride_bytes must be multiples of 16 bytes");
+        if (num_grads > 1 && grad_stride_bytes < gbytes) return fail(DCASGD_EINVAL, "dcasgd_apply_log: grad_stride_bytes smaller than one gradient");
+        if ((rc = check_foreign(c, grad_pool, (uint64_t)(num_grads - 1) * grad_stride_bytes + gbytes, "grad_pool"))) return rc;
+    }
+
+    if (window_k == 1) {
+        for (uint64_t r = 0; r < count; ++r) {
+            if (ev[r].kind == DCASGD_PULL) rc = launch_pull(s, ev[r].worker, nullptr);
+            else rc = launch_push(s, ev[r].worker, static_cast<const char*>(grad_pool) + (uint64_t)ev[r].grad_id * grad_stride_bytes, ev[r].eta);
+            if (rc) return rc;
+        }
+        return DCASGD_OK;
+    }
+
+    try {
+        WindowCompiler wc(c.num_workers);
+        dcasgd_window_program wp;
+        uint64_t r = 0;
+        while (r < count) {
+            if ((rc = wc.compile(ev + r, count - r, window_k, c.eta, &wp))) return rc;
+            if ((rc = launch_window(s, wp, grad_pool, grad_stride_bytes))) return rc;
+            r += wp.n_records;
+        }
+    } catch (const std::bad_alloc&) {
+        return fail(DCASGD_ENOMEM, "dcasgd_apply_log: out of host memory");
+    }
+    return DCASGD_OK;
+}
+
+int dcasgd_destroy(dcasgd_server* s) {
+    delete s;
+    return DCASGD_OK;
+}
+
+int dcasgd_get_step(const dcasgd_server* s, uint64_t* t) {
+    if (!s || !t) return fail(DCASGD_EINVAL, "dcasgd_get_step: NULL argument");
+    *t = s->t;
+    return DCASGD_OK;
+}
+
+int dcasgd_set_step(dcasgd_server* s, uint64_t t) {
+    if (!s) return fail(DCASGD_EINVAL, "dcasgd_set_step: server is NULL");
+    s->t = t;
+    return DCASGD_OK;
+}
+
+int dcasgd_get_launch_count(const dcasgd_server* s, uint64_t* launches) {
+    if (!s || !launches) return fail(DCASGD_EINVAL, "dcasgd_get_launch_count: NULL argument");
+    *launches = s->launches;
+    return DCASGD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU checker on the same
+seeded inputs.  The library never fuses a multiply-add and uses IEEE sqrt and division, so the
+bar is equality of every bit of w, w_bak[m] and ms (the stated tolerance
+max|dw| <= 1e-5 (1+|w|) is asserted as well)."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_1609_08326_b200 import binding as B
+from paper_1609_08326_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+PULL, PUSH = B.PULL, B.PUSH
+
+
+def small_workload(n, adaptive, bf16, M=3, pushes=24, G=6, seed=1, **kw):
+    return synth.Workload(name="t", n=n, M=M, pushes=pushes, adaptive=adaptive, bf16_grad=bf16, eta=0.1,
+                          lam=2.0 if adaptive else 0.04, mu=0.95 if adaptive else 0.0, eps=1e-7 if adaptive else 0.0,
+                          num_grads=G, nseg=3 if n >= 30 else 1, sigma_lo_exp=-4, sigma_hi_exp=-1, seed=seed, **kw)
+
+
+SIZES = [1, 2, 3, 4, 5, 127, 128, 129, 1023, 1024, 2049, 100_003, 272_474]
+
+
+@pytest.mark.parametrize("n", SIZES)
+@pytest.mark.parametrize("adaptive", [False, True])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_single_messages(n, adaptive, bf16):
+    """dcasgd_pull / dcasgd_push one message at a time, ragged sizes (n mod 4 in 0..3, below,
+    at and above a CTA's span)."""
+    import torch
+    wl = small_workload(n, adaptive, bf16)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+    dpool = U.to_device(pool)
+    out_w = torch.empty(n, dtype=torch.float32, device="cuda")
+    for r in ev:
+        m = int(r["worker"])
+        if r["kind"] == PULL:
+            gpu.pull(m, out_w)
+            cpu.pull(m)
+            assert np.array_equal(out_w.cpu().numpy(), cpu.w)          # the model sent back to the worker
+        else:
+            gpu.push(m, dpool[int(r["grad_id"])], float(r["eta"]))
+            cpu.push(m, pool[int(r["grad_id"]), :n], float(r["eta"]))
+    U.assert_state_equal(gpu, cpu)
+    assert gpu.launches == 1 + len(ev)
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 8, 32, 1000])
+@pytest.mark.parametrize("n", [5, 1023, 50_001])
+@pytest.mark.parametrize("adaptive,bf16", [(False, False), (True, False), (False, True), (True, True)])
+def test_apply_log_every_window_size(K, n, adaptive, bf16):
+    wl = small_workload(n, adaptive, bf16, M=8, pushes=150, G=12, seed=K)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+    gpu.apply_log(ev, U.to_device(pool), K)
+    cpu.replay(ev, np.ascontiguousarray(pool[:, :n]))
+    U.assert_state_equal(gpu, cpu, what=f"K={K} ")
+    if K == 1:
+        assert gpu.launches == 1 + len(ev)
+    else:
+        assert 2 <= gpu.launches <= 1 + -(-len(ev) // 2) + 2
+
+
+@pytest.mark.parametrize("proto,order", [(synth.PROTO_TAU0, synth.ORDER_UNIFORM), (synth.PROTO_SYNC, synth.ORDER_UNIFORM),
+                                         (synth.PROTO_ASYNC, synth.ORDER_ZIPF), (synth.PROTO_ASYNC, synth.ORDER_ROUND_ROBIN_JITTER)])
+def test_other_logs(proto, order):
+    wl = small_workload(4099, True, False, M=12, pushes=240, G=7, proto=proto, order=order, order_param=1.2)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    for K in (1, 16, 64):
+        gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+        gpu.apply_log(ev, dpool, K)
+        cpu.replay(ev, np.ascontiguousarray(pool[:, : wl.n]))
+        U.assert_state_equal(gpu, cpu)
+
+
+def test_record_soup_and_limits():
+    """Arbitrary records (repeated pulls, pushes with no pull, per-record eta, default eta), and
+    logs that overflow a window's slots, pushes and stores."""
+    rng = np.random.default_rng(3)
+    M, G, n = 40, 5, 777
+    logs = []
+    for _ in range(6):
+        recs = []
+        for _ in range(int(rng.integers(1, 200))):
+            if rng.random() < 0.55:
+                recs.append((PUSH, int(rng.integers(M)), int(rng.integers(G)), float(rng.choice([-1.0, 0.05, 0.2]))))
+            else:
+                recs.append((PULL, int(rng.integers(M))))
+        logs.append(synth.make_log(recs))
+    slots = []
+    for k in range(M):
+        slots += [(PUSH, k, k % G), (PULL, k)]
+    slots += [(PUSH, k, k % G) for k in range(M)]
+    logs.append(synth.make_log(slots))
+    logs.append(synth.make_log([(PUSH, 0, k % G) for k in range(300)]))
+    logs.append(synth.make_log([(PUSH, 0, 0)] + [(PULL, m % M) for m in range(250)] + [(PUSH, 3, 1)]))
+    wl = small_workload(n, True, False, M=M, G=G)
+    w0, pool = wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    for ev in logs:
+        for K in (7, 1000):
+            gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+            gpu.apply_log(ev, dpool, K)
+            cpu.replay(ev, np.ascontiguousarray(pool[:, :n]))
+            U.assert_state_equal(gpu, cpu)
+
+
+def test_apply_log_in_pieces_and_step_counter():
+    """Replaying 0..a then a..b equals replaying 0..b; t counts pushes only."""
+    wl = small_workload(30_001, True, False, M=5, pushes=100, G=9)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+    assert gpu.step == 0
+    a = 77
+    gpu.apply_log(ev[:a], dpool, 32)
+    assert gpu.step == int(np.sum(ev["kind"][:a] == PUSH))
+    gpu.apply_log(ev[a:a], dpool, 32)                       # empty log: no-op
+    gpu.apply_log(ev[a:], dpool, 5)
+    cpu.replay(ev, np.ascontiguousarray(pool[:, : wl.n]))
+    U.assert_state_equal(gpu, cpu)
+    assert gpu.step == 100
+
+
+def test_empty_model_and_side_stream():
+    import torch
+    wl = small_workload(0, True, False)
+    srv = B.Server(np.zeros(0, dtype=np.float32), 3, True, 0.1, 2.0, 0.95, 1e-7)
+    srv.pull(1)
+    srv.push(1, None)
+    srv.apply_log(wl.log(), torch.empty((6, 0), device="cuda"), 8, grad_stride_bytes=0, num_grads=6)
+    assert srv.step == 1 + wl.pushes and srv.launches == 0
+    # a server bound to a non-default stream
+    st = torch.cuda.Stream()
+    wl = small_workload(12_345, False, False)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    torch.cuda.synchronize()
+    gpu, cpu = U.gpu_server(wl, w0, stream=st), U.cpu_server(wl, w0)
+    gpu.apply_log(ev, dpool, 16)
+    st.synchronize()
+    cpu.replay(ev, np.ascontiguousarray(pool[:, : wl.n]))
+    U.assert_state_equal(gpu, cpu)
+
+
+def test_errors_leave_the_state_untouched():
+    import torch
+    wl = small_workload(1000, True, False, M=4)
+    w0, pool = wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    gpu = U.gpu_server(wl, w0)
+    torch.cuda.synchronize()
+    before = (gpu.w.clone(), gpu.w_bak_buf.clone(), gpu.ms.clone())
+    launches = gpu.launches
+
+    def expect(status, fn):
+        with pytest.raises(B.DcasgdError) as e:
+            fn()
+        assert e.value.status == status, e.value
+
+    expect(B.EWORKER, lambda: gpu.pull(4))
+    expect(B.EWORKER, lambda: gpu.push(9, dpool[0]))
+    expect(B.EINVAL, lambda: gpu.push(0, None))
+    expect(B.EALIGN, lambda: gpu.push(0, dpool[0].data_ptr() + 4))
+    expect(B.EINVAL, lambda: gpu.push(0, gpu.w))                                  # gradient aliases the model
+    expect(B.EINVAL, lambda: gpu.push(0, gpu.w_bak_buf[1024:]))
+    expect(B.EINVAL, lambda: gpu.push(0, dpool[0], float("nan")))
+    expect(B.EINVAL, lambda: gpu.pull(0, gpu.ms))
+    good = [(PUSH, 0, 0), (PULL, 0), (PUSH, 1, 1)]
+    for bad in ([(PUSH, 4, 0)], [(PUSH, 0, 6)], [(3, 0, 0)], [(PUSH, 0, 0, float("inf"))]):
+        for K in (1, 8):
+            expect(B.ELOG, lambda: gpu.apply_log(synth.make_log(good + bad), dpool, K))   # bad record at the END
+    expect(B.EINVAL, lambda: gpu.apply_log(synth.make_log(good), dpool, 0))
+    expect(B.EALIGN, lambda: gpu.apply_log(synth.make_log(good), dpool, 8, grad_stride_bytes=4004))
+    expect(B.EINVAL, lambda: gpu.apply_log(synth.make_log(good), gpu.w_bak_buf, 8, grad_stride_bytes=4096, num_grads=2))
+    torch.cuda.synchronize()
+    assert gpu.launches == launches and gpu.step == 0
+    for a, b in zip(before, (gpu.w, gpu.w_bak_buf, gpu.ms)):
+        assert torch.equal(a, b)
+    # host memory handed in as state is refused
+    host = torch.zeros(1000)
+    with pytest.raises(B.DcasgdError):
+        B.dcasgd_create(1000, 1, B.CONST, B.F32, 0.1, 0.04, 0, 0, host.data_ptr(), dpool.data_ptr(), 1024, None)
+
+
+def test_special_values_propagate_like_ieee():
+    """inf / nan / denormal / signed-zero inputs: same bits as the checker (no flush to zero)."""
+    n = 64
+    wl = small_workload(n, True, False, M=2, pushes=6, G=3)
+    w0 = wl.w0()
+    pool = U.host_pool(wl)
+    w0[:8] = [0.0, -0.0, 1e-40, -1e-40, np.inf, -np.inf, np.nan, 3e38]
+    pool[0, :8] = [1e-30, -1e-30, 1e-20, 0.0, 1.0, 1e20, 1.0, 3e38]
+    pool[1, 8:12] = [np.inf, np.nan, 1e-45, -0.0]
+    ev = wl.log()
+    for K in (1, 8):
+        gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+        gpu.apply_log(ev, U.to_device(pool), K)
+        with np.errstate(all="ignore"):
+            cpu.replay(ev, np.ascontiguousarray(pool[:, :n]))
+        U.assert_state_equal(gpu, cpu)
