@@ -109,21 +109,23 @@ class Server:
 
     def replay(self, ev: np.ndarray, grads: np.ndarray) -> None:
         """Apply a log serially.  `grads` is a [G][n] array (float32, uint16 bfloat16 patterns,
-        or float64 for a float64 server)."""
+        or float64 for a float64 server); rows may be strided (a column slice of a wider pool)."""
         assert ev.dtype.itemsize == 16 and ev.flags.c_contiguous
-        assert grads.ndim == 2 and grads.shape[1] == self.n and grads.flags.c_contiguous
+        assert grads.ndim == 2 and grads.shape[1] == self.n
+        assert grads.strides[1] == grads.itemsize and grads.strides[0] % grads.itemsize == 0
         G = grads.shape[0]
+        stride = grads.strides[0] // grads.itemsize
         if self.suf == "f32":
             assert grads.dtype in (np.float32, np.uint16)
             rc = self.L.oracle_replay_f32(self.n, self.M, int(self.adaptive), self.eta, self.lam,
                                           self.mu, self.eps, _ptr(self.w), _ptr(self.w_bak),
-                                          _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), self.n, G,
+                                          _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), stride, G,
                                           int(grads.dtype == np.uint16), C.addressof(self.t))
         else:
             assert grads.dtype == np.float64
             rc = self.L.oracle_replay_f64(self.n, self.M, int(self.adaptive), self.eta, self.lam,
                                           self.mu, self.eps, _ptr(self.w), _ptr(self.w_bak),
-                                          _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), self.n, G,
+                                          _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), stride, G,
                                           C.addressof(self.t))
         if rc != 0:
             raise ValueError(f"oracle rejected the log (code {rc})")
