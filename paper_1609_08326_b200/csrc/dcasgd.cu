@@ -121,13 +121,16 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     std::memset(&p, 0, sizeof p);
     p.n_pushes = wp.n_pushes;
     p.n_slots = wp.n_slots;
+    p.save_slot0 = (int8_t)wp.save_slot[0];
+    p.store_end0 = (uint16_t)wp.store_begin[1];
     for (uint32_t j = 0; j < wp.n_pushes; ++j) {
-        p.grad_id[j] = wp.grad_id[j];
-        p.eta[j] = wp.eta[j];
-        p.src[j] = wp.src[j];
+        Step& st = p.step[j];
+        st.grad_id = wp.grad_id[j];
+        st.eta = wp.eta[j];
+        st.src = wp.src[j];
+        st.save_slot = (int8_t)wp.save_slot[j + 1];
+        st.store_end = (uint16_t)wp.store_begin[j + 2];
     }
-    for (uint32_t j = 0; j <= wp.n_pushes; ++j) p.save_slot[j] = (int8_t)wp.save_slot[j];
-    for (uint32_t j = 0; j <= wp.n_pushes + 1; ++j) p.store_begin[j] = (uint8_t)wp.store_begin[j];
     for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_worker[k] = (uint16_t)wp.store_worker[k];
     ReplayArgs a;
     a.w = c.w;
@@ -139,7 +142,7 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.n = c.n;
     a.h = s->h;
     const unsigned grid = blocks_for(c.n, 1);
-    const size_t smem = (size_t)wp.n_slots * kThreads * sizeof(float4);
+    const size_t smem = replay_smem_bytes(wp.n_slots);
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
     if (ad && bf)       k_replay<true, true><<<grid, kThreads, smem, s->stream>>>(a, p);
     else if (ad)        k_replay<true, false><<<grid, kThreads, smem, s->stream>>>(a, p);
@@ -151,7 +154,7 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
 template <class K>
 cudaError_t allow_slots(K kernel) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                DCASGD_MAX_WINDOW_SLOTS * kThreads * (int)sizeof(float4));
+                                (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS));
 }
 
 int check_server(const dcasgd_server* s, const char* fn) {
