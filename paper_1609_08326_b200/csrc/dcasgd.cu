@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -17,6 +18,7 @@ struct dcasgd_server {
     Hyper h;
     cudaStream_t stream;
     int device;
+    int replay_vecs;     // 16-byte vectors per thread in the fused replay kernel (1 or 2)
     uint64_t t;          // pushes applied (Algorithm 2's t)
     uint64_t launches;   // kernels launched through this handle
 };
@@ -141,20 +143,30 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.grad_stride_bytes = grad_stride_bytes;
     a.n = c.n;
     a.h = s->h;
-    const unsigned grid = blocks_for(c.n, 1);
-    const size_t smem = replay_smem_bytes(wp.n_slots);
+    const int V = s->replay_vecs;
+    const unsigned grid = blocks_for(c.n, V);
+    const size_t smem = replay_smem_bytes(wp.n_slots, V);
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
-    if (ad && bf)       k_replay<true, true><<<grid, kThreads, smem, s->stream>>>(a, p);
-    else if (ad)        k_replay<true, false><<<grid, kThreads, smem, s->stream>>>(a, p);
-    else if (bf)        k_replay<false, true><<<grid, kThreads, smem, s->stream>>>(a, p);
-    else                k_replay<false, false><<<grid, kThreads, smem, s->stream>>>(a, p);
+#define DCASGD_LAUNCH_REPLAY(AD, BF)                                                         \
+    do {                                                                                     \
+        if (V == 2) k_replay<AD, BF, 2><<<grid, kThreads, smem, s->stream>>>(a, p);          \
+        else        k_replay<AD, BF, 1><<<grid, kThreads, smem, s->stream>>>(a, p);          \
+    } while (0)
+    if (ad && bf)       DCASGD_LAUNCH_REPLAY(true, true);
+    else if (ad)        DCASGD_LAUNCH_REPLAY(true, false);
+    else if (bf)        DCASGD_LAUNCH_REPLAY(false, true);
+    else                DCASGD_LAUNCH_REPLAY(false, false);
+#undef DCASGD_LAUNCH_REPLAY
     return after_launch(s, "window replay kernel");
 }
 
-template <class K>
-cudaError_t allow_slots(K kernel) {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS));
+template <bool AD, bool BF>
+cudaError_t allow_slots() {
+    cudaError_t e = cudaFuncSetAttribute(k_replay<AD, BF, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 1));
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(k_replay<AD, BF, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 2));
 }
 
 int check_server(const dcasgd_server* s, const char* fn) {
@@ -237,8 +249,8 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
                 return fail(DCASGD_EINVAL, "dcasgd_create: %s lives on device %d, current device is %d", names[i], at.device, dev);
         }
     }
-    if ((e = allow_slots(k_replay<false, false>)) != cudaSuccess || (e = allow_slots(k_replay<false, true>)) != cudaSuccess ||
-        (e = allow_slots(k_replay<true, false>)) != cudaSuccess || (e = allow_slots(k_replay<true, true>)) != cudaSuccess)
+    if ((e = allow_slots<false, false>()) != cudaSuccess || (e = allow_slots<false, true>()) != cudaSuccess ||
+        (e = allow_slots<true, false>()) != cudaSuccess || (e = allow_slots<true, true>()) != cudaSuccess)
         return cuda_fail("dcasgd_create: cudaFuncSetAttribute", e);
 
     dcasgd_server* s = new (std::nothrow) dcasgd_server;
@@ -252,6 +264,10 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->device = dev;
     s->t = 0;
     s->launches = 0;
+    // one vector per thread measured faster on B200 (higher occupancy beats the saved uniform work);
+    // DCASGD_REPLAY_VECS=2 selects the two-vector kernel for experiments
+    s->replay_vecs = 1;
+    if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) s->replay_vecs = std::atoi(v) == 2 ? 2 : 1;
     if (c.n) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
