@@ -67,3 +67,32 @@ def assert_state_equal(gpu: B.Server, cpu: oracle.Server, idx: np.ndarray | None
         assert np.all(tol_ok | same), f"{what}{name}: outside tolerance"
         assert np.all(same), f"{what}{name}: {np.count_nonzero(~same)} of {same.size} elements differ in bits"
     assert gpu.step == cpu.step
+
+
+def cpu_replay_ranges(wl: synth.Workload, ev: np.ndarray, w0: np.ndarray, pool: np.ndarray, threads: int):
+    """The checker's serial replay over the full vector, its unchanged replay function called on
+    disjoint element ranges from several host threads (elements never interact).  Returns the
+    per-range servers and their bounds."""
+    import threading
+    bounds = np.linspace(0, wl.n, threads + 1).astype(np.int64)
+    servers = [cpu_server(wl, w0[lo:hi]) for lo, hi in zip(bounds[:-1], bounds[1:])]
+    ths = [threading.Thread(target=s.replay, args=(ev, pool[:, lo:hi]))
+           for s, lo, hi in zip(servers, bounds[:-1], bounds[1:])]
+    for t in ths:
+        t.start()
+    for t in ths:
+        t.join()
+    return servers, bounds
+
+
+def assert_ranges_equal(gpu: B.Server, servers, bounds) -> None:
+    import torch
+    torch.cuda.synchronize()
+    for s, lo, hi in zip(servers, bounds[:-1], bounds[1:]):
+        pairs = [("w", gpu.w[lo:hi], s.w), ("w_bak", gpu.w_bak[:, lo:hi], s.w_bak)]
+        if s.ms is not None:
+            pairs.append(("ms", gpu.ms[lo:hi], s.ms))
+        for name, got, want in pairs:
+            got = got.cpu().numpy()
+            assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), f"{name}[{lo}:{hi}] differs"
+        assert gpu.step == s.step
