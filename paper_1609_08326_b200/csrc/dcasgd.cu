@@ -260,6 +260,9 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->h.mu = adaptive ? c.mu : 0.0f;
     s->h.omm = 1.0f - s->h.mu;
     s->h.eps = adaptive ? c.eps : 0.0f;
+    const float al = std::fabs(c.lambda);
+    s->h.fast = (al >= 0x1p-60f && al < 0x1p60f) ? 1u : 0u;
+    if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) s->h.fast = 0u; }
     s->stream = static_cast<cudaStream_t>(c.stream);
     s->device = dev;
     s->t = 0;

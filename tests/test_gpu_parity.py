@@ -205,3 +205,23 @@ def test_special_values_propagate_like_ieee():
         with np.errstate(all="ignore"):
             cpu.replay(ev, np.ascontiguousarray(pool[:, :n]))
         U.assert_state_equal(gpu, cpu)
+
+
+@pytest.mark.parametrize("lam,eps", [(2.0, 0.0), (0.0, 1e-7), (-0.0, 1e-7), (-2.0, 1e-7), (1e25, 1e-7), (3e-30, 0.0),
+                                     (2.0, 1e-38), (0.04, 1e30)])
+def test_adaptive_lambda_routes(lam, eps):
+    """lambda_t = lambda_0 / sqrt(ms + eps) takes a branch-free exact route when ms + eps lies in
+    [2^-100, 2^100) and |lambda_0| in [2^-60, 2^60), and the guarded IEEE route otherwise (zero,
+    denormal, huge, non-finite).  Both must give the checker's bits; mixed within one vector."""
+    n = 4096
+    wl = small_workload(n, True, False, M=4, pushes=40, G=8).scaled(lam=lam, eps=eps)
+    w0, pool, ev = wl.w0(), U.host_pool(wl), wl.log()
+    rng = np.random.default_rng(5)
+    scale = rng.choice([0.0, 1e-30, 1e-22, 1e-12, 1e-3, 1.0, 1e12, 1e18], size=n).astype(np.float32)
+    pool[:, :n] = (pool[:, :n] / np.float32(1e-2)) * scale          # every magnitude class in every vector
+    for K in (1, 32):
+        gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+        gpu.apply_log(ev, U.to_device(pool), K)
+        with np.errstate(all="ignore"):
+            cpu.replay(ev, pool[:, :n])
+        U.assert_state_equal(gpu, cpu, what=f"lam={lam} eps={eps} K={K} ")
