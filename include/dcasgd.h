@@ -134,6 +134,16 @@ const char *dcasgd_last_error(void);        /* never NULL; valid until the threa
 const char *dcasgd_status_string(int status);
 uint32_t dcasgd_version(void);
 
+/* Diagnostic, no counterpart in the paper.  For the adaptive variant the kernels compute
+ * lambda_t = lambda_0 / sqrt(s), s = ms + eps, on a branch-free route (packed FMAs, one Newton
+ * correction for the root, Markstein-style corrected quotient) when s is in [2^-100, 2^100) and
+ * |lambda_0| in [2^-60, 2^60), and with the compiler's guarded IEEE sqrt and division otherwise.
+ * This call runs both routes on EVERY binary32 value s in [s_first, s_last] for the given
+ * lambda_0 and ADDS the number of inputs on which their bits differ to *mismatches_dev (device,
+ * 8 bytes, 8-byte aligned, zeroed by the caller).  Enqueued on `stream`; allocates nothing.
+ * The expected count is 0 for every admissible argument. */
+int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, void *stream, uint64_t *mismatches_dev);
+
 /* ---- window compiler (host only; no CUDA call) -------------------------------------------
  * What dcasgd_apply_log does to a window before launching, exposed so that it can be
  * inspected and tested without a GPU.  A window of the log becomes a list of STEPS.  Step 0 has

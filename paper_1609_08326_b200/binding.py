@@ -29,7 +29,7 @@ MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
 # every symbol include/dcasgd.h declares
 SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
            "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_last_error",
-           "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window"]
+           "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window", "dcasgd_check_adaptive_lambda"]
 
 
 class Config(C.Structure):
@@ -76,6 +76,8 @@ def lib() -> C.CDLL:
         L.dcasgd_set_step.argtypes = [vp, u64]
         L.dcasgd_get_launch_count.argtypes = [vp, C.POINTER(u64)]
         L.dcasgd_compile_window.argtypes = [vp, u64, u32, u32, C.c_float, C.POINTER(WindowProgram)]
+        L.dcasgd_check_adaptive_lambda.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp]
+        L.dcasgd_check_adaptive_lambda.restype = C.c_int
         for name in ("dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
                      "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_compile_window"):
             getattr(L, name).restype = C.c_int
@@ -171,6 +173,12 @@ def dcasgd_compile_window(ev, num_workers, window_k, default_eta=0.0) -> WindowP
     return out
 
 
+def dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, mismatches_dev, stream=None) -> None:
+    """Adds to the device counter the number of s in [s_first, s_last] on which the two routes
+    of lambda_0 / sqrt(s) differ (expected: 0)."""
+    _check(lib().dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, stream, _ptr(mismatches_dev)))
+
+
 def plan_log(ev, num_workers, window_k, default_eta=0.0) -> list[WindowProgram]:
     """All windows of a log, as dcasgd_apply_log would cut them."""
     out, r = [], 0
@@ -179,6 +187,50 @@ def plan_log(ev, num_workers, window_k, default_eta=0.0) -> list[WindowProgram]:
         out.append(p)
         r += p.n_records
     return out
+
+
+def apply_log_from_host(h, ev, host_pool, dev_pool, window_k, copy_stream, chunk: int = 8) -> int:
+    """dcasgd_apply_log for a gradient pool that still sits in (pinned) host memory.
+
+    `host_pool` and `dev_pool` are [G][row] torch tensors of the same shape and dtype.  The pool
+    buffers are copied to the device on `copy_stream` in the order in which the log first uses
+    them, `chunk` buffers per event, and each piece of the log is enqueued (on the current
+    stream, which must be the server's) as soon as the buffers it names have arrived, so the
+    transfer overlaps the replay of the earlier pieces.  Results equal one dcasgd_apply_log call
+    on a resident pool.  Returns the number of host->device bytes enqueued."""
+    import torch
+    ev = np.ascontiguousarray(ev)
+    G = host_pool.shape[0]
+    stride = dev_pool.stride(0) * dev_pool.element_size()
+    push_idx = np.flatnonzero(ev["kind"] == PUSH)
+    gids = ev["grad_id"][push_idx]
+    order, first_rec = [], []                         # buffers in first-use order, record of first use
+    seen = set()
+    for r, g in zip(push_idx.tolist(), gids.tolist()):
+        if g not in seen:
+            seen.add(g)
+            order.append(g)
+            first_rec.append(r)
+            if len(seen) == G:
+                break
+    main = torch.cuda.current_stream()
+    copy_stream.wait_stream(main)                     # the device pool may still be read by earlier work
+    start, nbytes = 0, 0
+    for c in range(0, len(order), chunk):
+        with torch.cuda.stream(copy_stream):
+            for g in order[c:c + chunk]:
+                dev_pool[g].copy_(host_pool[g], non_blocking=True)
+                nbytes += host_pool[g].numel() * host_pool.element_size()
+            arrived = torch.cuda.Event()
+            arrived.record(copy_stream)
+        nxt = c + chunk
+        end = first_rec[nxt] if nxt < len(order) else len(ev)
+        main.wait_event(arrived)
+        dcasgd_apply_log(h, ev[start:end], dev_pool, stride, G, window_k)
+        start = end
+    if start < len(ev):
+        dcasgd_apply_log(h, ev[start:], dev_pool, stride, G, window_k)
+    return nbytes
 
 
 # ---------------------------------------------------------------- convenience wrapper

@@ -373,6 +373,22 @@ int dcasgd_set_step(dcasgd_server* s, uint64_t t) {
     return DCASGD_OK;
 }
 
+int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, void* stream, uint64_t* mismatches_dev) {
+    if (!mismatches_dev) return fail(DCASGD_EINVAL, "dcasgd_check_adaptive_lambda: mismatches_dev is NULL");
+    const float al = std::fabs(lambda0);
+    if (!(al >= 0x1p-60f && al < 0x1p60f)) return fail(DCASGD_EINVAL, "dcasgd_check_adaptive_lambda: |lambda0| must be in [2^-60, 2^60)");
+    if (!(s_first >= 0x1p-100f && s_last < 0x1p100f && s_first <= s_last))
+        return fail(DCASGD_EINVAL, "dcasgd_check_adaptive_lambda: need 2^-100 <= s_first <= s_last < 2^100");
+    uint32_t b0, b1;
+    std::memcpy(&b0, &s_first, 4);
+    std::memcpy(&b1, &s_last, 4);
+    k_check_lambda<<<148 * 8, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        lambda0, b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("lambda self-check kernel", e);
+    return DCASGD_OK;
+}
+
 int dcasgd_get_launch_count(const dcasgd_server* s, uint64_t* launches) {
     if (!s || !launches) return fail(DCASGD_EINVAL, "dcasgd_get_launch_count: NULL argument");
     *launches = s->launches;

@@ -225,3 +225,36 @@ def test_adaptive_lambda_routes(lam, eps):
         with np.errstate(all="ignore"):
             cpu.replay(ev, pool[:, :n])
         U.assert_state_equal(gpu, cpu, what=f"lam={lam} eps={eps} K={K} ")
+
+
+def test_adaptive_lambda_branch_free_route_is_exact_for_every_s():
+    """Exhaustive: for several lambda_0 (the paper's 2 and 0.04 among them) the branch-free
+    lambda_0 / sqrt(s) equals the IEEE sqrt-then-divide on all 1.68e9 binary32 values of s in
+    [2^-100, 2^100)."""
+    import torch
+    counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+    last = float(np.nextafter(np.float32(2.0 ** 100), np.float32(0)))
+    for lam0 in (2.0, 0.04, 1.0, -2.0, 0.3, 1.9999999, 7.7e-12, 3.3e9):
+        B.dcasgd_check_adaptive_lambda(lam0, 2.0 ** -100, last, counter)
+    torch.cuda.synchronize()
+    assert int(counter.item()) == 0
+    for bad in (lambda: B.dcasgd_check_adaptive_lambda(0.0, 1.0, 2.0, counter),
+                lambda: B.dcasgd_check_adaptive_lambda(2.0, 0.0, 2.0, counter),
+                lambda: B.dcasgd_check_adaptive_lambda(2.0, 1.0, 2.0, None)):
+        with pytest.raises(B.DcasgdError):
+            bad()
+
+
+def test_apply_log_from_host_overlapped_copies():
+    """The pool arrives from pinned host memory on a copy stream while earlier pieces of the log
+    replay: same bits as the checker (and as a resident pool)."""
+    import torch
+    wl = small_workload(200_003, True, False, M=6, pushes=300, G=20)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    host = torch.from_numpy(pool).pin_memory()
+    dev = torch.full(host.shape, float("nan"), device="cuda")          # nothing resident beforehand
+    gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+    nbytes = B.apply_log_from_host(gpu.h, ev, host, dev, 32, torch.cuda.Stream(), chunk=3)
+    assert nbytes == host.numel() * 4
+    cpu.replay(ev, pool[:, : wl.n])
+    U.assert_state_equal(gpu, cpu)
