@@ -65,6 +65,10 @@ typedef enum {
 enum { DCASGD_CONST = 0, DCASGD_ADAPTIVE = 1 }; /* DC-ASGD-c / DC-ASGD-a (Section 6) */
 enum { DCASGD_F32 = 0, DCASGD_BF16 = 1 };       /* storage type of pushed gradients */
 enum { DCASGD_PULL = 0, DCASGD_PUSH = 1 };      /* the two messages of Algorithm 2 */
+/* dcasgd_config.flags.  DCASGD_RESUME: w, w_bak and ms already hold a saved server state (a
+ * checkpoint the caller copied into them): dcasgd_create leaves them as they are instead of
+ * running "Initialize"; restore t with dcasgd_set_step. */
+enum { DCASGD_RESUME = 1u };
 
 typedef struct {
   uint64_t n;            /* number of parameters; 0 is allowed (every call is then a no-op) */
@@ -75,6 +79,7 @@ typedef struct {
   float lambda;          /* lambda (constant variant) or lambda_0 (adaptive variant); any finite value */
   float mu;              /* the paper's moving-average constant "m", in [0,1); adaptive only */
   float eps;             /* >= 0; the paper uses 1e-7; adaptive only */
+  uint32_t flags;        /* 0, or DCASGD_RESUME */
   float *w;              /* device, n floats, 16-byte aligned; holds w_0 on entry */
   float *w_bak;          /* device, num_workers slabs of w_bak_stride floats, 16-byte aligned */
   uint64_t w_bak_stride; /* floats between slabs: >= n and a multiple of 4 */
@@ -91,7 +96,7 @@ typedef struct {
   float eta;        /* PUSH: learning rate of this update, < 0 = the server's default; PULL: ignored */
 } dcasgd_event;
 
-/* Algorithm 2, "Initialize": t = 0, w_bak[m] = w for every m, ms = 0.
+/* Algorithm 2, "Initialize": t = 0, w_bak[m] = w for every m, ms = 0 (skipped with DCASGD_RESUME).
  * cfg (host) is copied.  *out receives the handle.  w, w_bak, ms must not overlap. */
 int dcasgd_create(const dcasgd_config *cfg, dcasgd_server **out);
 

@@ -24,6 +24,7 @@ OK, EINVAL, EWORKER, EALIGN, ELOG, ECUDA, ENOMEM = range(7)
 CONST, ADAPTIVE = 0, 1
 F32, BF16 = 0, 1
 PULL, PUSH = 0, 1
+RESUME = 1
 MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
 
 # every symbol include/dcasgd.h declares
@@ -35,7 +36,7 @@ SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "d
 class Config(C.Structure):
     _fields_ = [("n", C.c_uint64), ("num_workers", C.c_uint32), ("variant", C.c_uint32),
                 ("grad_dtype", C.c_uint32), ("eta", C.c_float), ("lambda_", C.c_float),
-                ("mu", C.c_float), ("eps", C.c_float), ("w", C.c_void_p), ("w_bak", C.c_void_p),
+                ("mu", C.c_float), ("eps", C.c_float), ("flags", C.c_uint32), ("w", C.c_void_p), ("w_bak", C.c_void_p),
                 ("w_bak_stride", C.c_uint64), ("ms", C.c_void_p), ("stream", C.c_void_p)]
 
 
@@ -116,8 +117,8 @@ def _ptr(x) -> int | None:
 # ---------------------------------------------------------------- the C calls, one to one
 
 def dcasgd_create(n, num_workers, variant, grad_dtype, eta, lam, mu, eps, w, w_bak, w_bak_stride,
-                  ms, stream=None) -> int:
-    cfg = Config(n, num_workers, variant, grad_dtype, eta, lam, mu, eps, _ptr(w), _ptr(w_bak),
+                  ms, stream=None, flags=0) -> int:
+    cfg = Config(n, num_workers, variant, grad_dtype, eta, lam, mu, eps, flags, _ptr(w), _ptr(w_bak),
                  w_bak_stride, _ptr(ms), stream)
     h = C.c_void_p()
     _check(lib().dcasgd_create(C.byref(cfg), C.byref(h)))
@@ -244,23 +245,37 @@ class Server:
     """Owns the torch tensors a server borrows (w, w_bak, ms) and the handle."""
 
     def __init__(self, w0, num_workers: int, adaptive: bool, eta: float, lam: float, mu: float = 0.0,
-                 eps: float = 0.0, bf16_grad: bool = False, device="cuda", stream=None):
+                 eps: float = 0.0, bf16_grad: bool = False, device="cuda", stream=None, state: dict | None = None):
+        """`state` (from state_dict()) resumes a saved server instead of initialising from w0."""
         import torch
         self.torch = torch
         self.device = torch.device(device)
-        w0 = torch.as_tensor(w0, dtype=torch.float32).reshape(-1)
+        w0 = torch.as_tensor(w0 if state is None else state["w"], dtype=torch.float32).reshape(-1)
         self.n = int(w0.numel())
         self.M = int(num_workers)
         self.stride = padded_stride(self.n)
         self.w = w0.to(self.device, copy=True).contiguous()
         self.w_bak_buf = torch.empty(self.M * self.stride, dtype=torch.float32, device=self.device)
         self.ms = torch.empty(self.n, dtype=torch.float32, device=self.device) if adaptive else None
+        if state is not None:
+            self.w_bak_buf.view(self.M, self.stride)[:, : self.n].copy_(state["w_bak"])
+            if adaptive:
+                self.ms.copy_(state["ms"])
         self.bf16_grad = bool(bf16_grad)
         self.stream = stream
         s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(self.device).cuda_stream
         with torch.cuda.device(self.device):
             self.h = dcasgd_create(self.n, self.M, ADAPTIVE if adaptive else CONST, BF16 if bf16_grad else F32,
-                                   eta, lam, mu, eps, self.w, self.w_bak_buf, self.stride, self.ms, s)
+                                   eta, lam, mu, eps, self.w, self.w_bak_buf, self.stride, self.ms, s,
+                                   flags=RESUME if state is not None else 0)
+        if state is not None:
+            dcasgd_set_step(self.h, int(state["t"]))
+
+    def state_dict(self) -> dict:
+        """The whole server state (w, every backup, MeanSquare, t) as host copies: a checkpoint."""
+        self.torch.cuda.synchronize(self.device)
+        return {"w": self.w.cpu(), "w_bak": self.w_bak.cpu(), "ms": None if self.ms is None else self.ms.cpu(),
+                "t": self.step}
 
     @property
     def w_bak(self):

@@ -207,6 +207,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
         return fail(DCASGD_EINVAL, "dcasgd_create: num_workers must be 1..65535 (got %u)", c.num_workers);
     if (c.variant > DCASGD_ADAPTIVE) return fail(DCASGD_EINVAL, "dcasgd_create: unknown variant %u", c.variant);
     if (c.grad_dtype > DCASGD_BF16) return fail(DCASGD_EINVAL, "dcasgd_create: unknown grad_dtype %u", c.grad_dtype);
+    if (c.flags & ~(uint32_t)DCASGD_RESUME) return fail(DCASGD_EINVAL, "dcasgd_create: unknown flags 0x%x", c.flags);
     if (!std::isfinite(c.eta) || c.eta < 0.0f) return fail(DCASGD_EINVAL, "dcasgd_create: eta must be finite and >= 0");
     if (!std::isfinite(c.lambda)) return fail(DCASGD_EINVAL, "dcasgd_create: lambda must be finite");
     const bool adaptive = c.variant == DCASGD_ADAPTIVE;
@@ -271,7 +272,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     // DCASGD_REPLAY_VECS=2 selects the two-vector kernel for experiments
     s->replay_vecs = 1;
     if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) s->replay_vecs = std::atoi(v) == 2 ? 2 : 1;
-    if (c.n) {
+    if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
         const int rc = after_launch(s, "init kernel");

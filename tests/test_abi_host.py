@@ -34,7 +34,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_layouts_match_the_header():
     assert C.sizeof(B.Config) == 80
-    assert B.Config.w.offset == 40 and B.Config.w_bak_stride.offset == 56 and B.Config.ms.offset == 64 and B.Config.stream.offset == 72
+    assert B.Config.flags.offset == 36 and B.Config.w.offset == 40 and B.Config.w_bak_stride.offset == 56 and B.Config.ms.offset == 64 and B.Config.stream.offset == 72
     assert synth.EVENT_DTYPE.itemsize == 16
     words = 6 + 3 * B.MAX_WINDOW_PUSHES + (B.MAX_WINDOW_PUSHES + 1) + (B.MAX_WINDOW_PUSHES + 2) + B.MAX_WINDOW_STORES
     assert C.sizeof(B.WindowProgram) == 4 * words
@@ -46,14 +46,14 @@ def test_struct_layouts_match_the_header():
 def _create(**kw):
     # fake but well-formed addresses: validation must fail before any of them is dereferenced
     args = dict(n=1000, num_workers=4, variant=B.ADAPTIVE, grad_dtype=B.F32, eta=0.1, lam=2.0, mu=0.95,
-                eps=1e-7, w=0x10000, w_bak=0x20000, w_bak_stride=1000, ms=0x40000, stream=None)
+                eps=1e-7, flags=0, w=0x10000, w_bak=0x20000, w_bak_stride=1000, ms=0x40000, stream=None)
     args.update(kw)
     return B.dcasgd_create(**args)
 
 
 @pytest.mark.parametrize("kw,status", [
     (dict(num_workers=0), B.EINVAL), (dict(num_workers=70000), B.EINVAL),
-    (dict(variant=2), B.EINVAL), (dict(grad_dtype=2), B.EINVAL),
+    (dict(variant=2), B.EINVAL), (dict(grad_dtype=2), B.EINVAL), (dict(flags=2), B.EINVAL),
     (dict(eta=float("nan")), B.EINVAL), (dict(lam=float("inf")), B.EINVAL),
     (dict(mu=1.0), B.EINVAL), (dict(mu=-0.1), B.EINVAL), (dict(eps=-1e-7), B.EINVAL),
     (dict(ms=None), B.EINVAL), (dict(variant=B.CONST), B.EINVAL),          # ms given to the constant variant

@@ -258,3 +258,37 @@ def test_apply_log_from_host_overlapped_copies():
     assert nbytes == host.numel() * 4
     cpu.replay(ev, pool[:, : wl.n])
     U.assert_state_equal(gpu, cpu)
+
+
+def test_checkpoint_and_resume():
+    """Replay 0..a, save the server state, resume a NEW server from the copy and replay a..b:
+    bit for bit the same as replaying 0..b in one go (and as the checker)."""
+    wl = small_workload(20_001, True, False, M=5, pushes=120, G=9)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    a = 101
+    first = U.gpu_server(wl, w0)
+    first.apply_log(ev[:a], dpool, 16)
+    ckpt = first.state_dict()
+    first.close()
+    del first
+    resumed = B.Server(None, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, wl.bf16_grad, state=ckpt)
+    assert resumed.step == ckpt["t"] == int(np.sum(ev["kind"][:a] == PUSH))
+    resumed.apply_log(ev[a:], dpool, 16)
+    cpu = U.cpu_server(wl, w0)
+    cpu.replay(ev, pool[:, : wl.n])
+    U.assert_state_equal(resumed, cpu)
+
+
+def test_delay_compensated_synchronous_rounds():
+    """Supplementary: rounds of M pushes against one shared snapshot with eta_hat / M, as a log."""
+    M = 8
+    wl = small_workload(33_333, False, False, M=M, pushes=M * 12, G=M * 12, proto=synth.PROTO_SYNC).scaled(eta=0.5 / M, lam=2.0)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    for K in (1, 2 * M, 64):
+        gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+        gpu.apply_log(ev, U.to_device(pool), K)
+        cpu.replay(ev, pool[:, : wl.n])
+        U.assert_state_equal(gpu, cpu)
+    (p,) = B.plan_log(ev[: 2 * M], M, 2 * M, wl.eta)
+    assert p.n_slots == 1 and p.n_snapshot_reads == 0 and p.n_stores == M      # one shared in-window snapshot

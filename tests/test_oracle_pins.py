@@ -288,9 +288,38 @@ def pin_f32_tracks_f64(L):
         assert np.all(np.abs(s32.w - s64.w) <= 1e-5 * (1 + np.abs(s64.w)))
 
 
+def pin_delay_compensated_ssgd(L):
+    """Supplementary, "Large mini-batch synchronous SGD with delay-compensated gradient": M
+    gradients all computed at w_t are applied one after another with eta_hat/M, each compensated
+    against the shared snapshot w_t.  Expressed as a log (all workers pull, then all push), the
+    checker must equal that recursion over the rationals; with lambda = 0 it is the plain
+    large-batch step w_t - eta_hat * mean(g)."""
+    rng = np.random.default_rng(21)
+    n, M, rounds = 4, 4, 2
+    eta_hat, lam = Fr(1, 2), Fr(2)
+    w0 = rng.integers(-16, 17, n) / 8.0
+    grads = rng.choice([-1.0, -0.5, 0.5, 1.0], size=(M * rounds, n))
+    ev = synth.event_log(M, M * rounds, synth.ORDER_UNIFORM, synth.PROTO_SYNC, M * rounds, float(eta_hat / M), seed=4)
+    for lam_ in (lam, Fr(0)):
+        s = oracle.Server(w0, M, False, float(eta_hat / M), float(lam_), dtype=np.float64, library=L)
+        s.replay(ev, np.ascontiguousarray(grads, dtype=np.float64))
+        w = [Fr(x) for x in w0]
+        pushes = ev[ev["kind"] == PUSH]
+        for r in range(rounds):
+            wt = list(w)                                  # the snapshot every worker pulled
+            gsum = [Fr(0)] * n
+            for rec in pushes[r * M:(r + 1) * M]:
+                g = [Fr(float(x)) for x in grads[int(rec["grad_id"])]]
+                w = [w[i] - eta_hat / M * (g[i] + lam_ * g[i] * g[i] * (w[i] - wt[i])) for i in range(n)]
+                gsum = [a + b for a, b in zip(gsum, g)]
+            if lam_ == 0:
+                assert w == [wt[i] - eta_hat * gsum[i] / M for i in range(n)]
+        assert [Fr(float(x)) for x in s.w] == w
+
+
 PINS = [pin_hand_constant, pin_closed_form_repeated, pin_hand_adaptive, pin_exact_rational_replay,
         pin_lambda0_is_asgd, pin_tau0_is_sgd, pin_meansquare_unrolled, pin_adaptive_lambda_definition,
-        pin_protocol, pin_bruteforce_f32, pin_f32_tracks_f64]
+        pin_protocol, pin_bruteforce_f32, pin_f32_tracks_f64, pin_delay_compensated_ssgd]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
