@@ -119,28 +119,28 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     s->t += wp.n_pushes;
     if (c.n == 0) return DCASGD_OK;
     if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
-    DevProgram p;
+    static thread_local DevProgram p;            // 4.6 KB: kept off the stack
     std::memset(&p, 0, sizeof p);
     p.n_pushes = wp.n_pushes;
     p.n_slots = wp.n_slots;
     p.save_slot0 = (int8_t)wp.save_slot[0];
-    p.store_end0 = (uint16_t)wp.store_begin[1];
+    p.store_end0 = (uint8_t)wp.store_begin[1];
     for (uint32_t j = 0; j < wp.n_pushes; ++j) {
-        Step& st = p.step[j];
-        st.grad_id = wp.grad_id[j];
-        st.eta = wp.eta[j];
-        st.src = wp.src[j];
-        st.save_slot = (int8_t)wp.save_slot[j + 1];
-        st.store_end = (uint16_t)wp.store_begin[j + 2];
+        FetchStep& f = p.fetch[j];
+        ApplyStep& ap = p.apply[j];
+        f.g_off = (uint64_t)wp.grad_id[j] * grad_stride_bytes;
+        ap.eta = wp.eta[j];
+        if (wp.src[j] >= 0) { ap.src_slot = -1; f.s_off = (uint64_t)wp.src[j] * c.w_bak_stride * 4; }
+        else                { ap.src_slot = (int8_t)(-(wp.src[j] + 1)); f.s_off = kNoMemorySnapshot; }
+        ap.save_slot = (int8_t)wp.save_slot[j + 1];
+        ap.store_end = (uint8_t)wp.store_begin[j + 2];
     }
-    for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_worker[k] = (uint16_t)wp.store_worker[k];
+    for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_off[k] = (uint64_t)wp.store_worker[k] * c.w_bak_stride * 4;
     ReplayArgs a;
     a.w = c.w;
     a.w_bak = c.w_bak;
     a.ms = c.ms;
     a.grad_pool = static_cast<const char*>(grad_pool);
-    a.stride = c.w_bak_stride;
-    a.grad_stride_bytes = grad_stride_bytes;
     a.n = c.n;
     a.h = s->h;
     const int V = s->replay_vecs;
