@@ -81,7 +81,8 @@ typedef struct {
   float eps;             /* >= 0; the paper uses 1e-7; adaptive only */
   uint32_t flags;        /* 0, or DCASGD_RESUME */
   float *w;              /* device, n floats, 16-byte aligned; holds w_0 on entry */
-  float *w_bak;          /* device, num_workers slabs of w_bak_stride floats, 16-byte aligned */
+  float *w_bak;          /* device, num_workers * w_bak_stride floats (every slab is padded to the stride;
+                            the padding may be overwritten), 16-byte aligned */
   uint64_t w_bak_stride; /* floats between slabs: >= n and a multiple of 4 */
   float *ms;             /* device, n floats, 16-byte aligned; NULL if and only if DCASGD_CONST */
   void *stream;          /* cudaStream_t; NULL is the legacy default stream */

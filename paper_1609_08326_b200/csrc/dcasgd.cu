@@ -56,7 +56,7 @@ int cuda_fail(const char* what, cudaError_t e) {
 int state_ranges(const dcasgd_config& c, Range out[3]) {
     int k = 0;
     out[k++] = range_of(c.w, c.n * 4, "w");
-    const uint64_t bak = c.n == 0 ? 0 : ((uint64_t)(c.num_workers - 1) * c.w_bak_stride + c.n) * 4;
+    const uint64_t bak = c.n == 0 ? 0 : (uint64_t)c.num_workers * c.w_bak_stride * 4;   // every slab is stride floats long
     out[k++] = range_of(c.w_bak, bak, "w_bak");
     if (c.ms) out[k++] = range_of(c.ms, c.n * 4, "ms");
     return k;
