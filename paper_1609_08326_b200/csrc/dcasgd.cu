@@ -268,10 +268,11 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->device = dev;
     s->t = 0;
     s->launches = 0;
-    // one vector per thread measured faster on B200 (higher occupancy beats the saved uniform work);
-    // DCASGD_REPLAY_VECS=2 selects the two-vector kernel for experiments
-    s->replay_vecs = 1;
-    if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) s->replay_vecs = std::atoi(v) == 2 ? 2 : 1;
+    // two vectors per thread (3 CTAs/SM, 3-stage ring) measured 4-6 % faster on B200 than one vector
+    // per thread (4 CTAs/SM, 5-stage ring): the per-push control work is shared by 8 elements;
+    // DCASGD_REPLAY_VECS=1 selects the one-vector kernel for experiments
+    s->replay_vecs = 2;
+    if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) s->replay_vecs = std::atoi(v) == 1 ? 1 : 2;
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
