@@ -268,11 +268,14 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->device = dev;
     s->t = 0;
     s->launches = 0;
-    // two vectors per thread (3 CTAs/SM, 3-stage ring) measured 4-6 % faster on B200 than one vector
-    // per thread (4 CTAs/SM, 5-stage ring): the per-push control work is shared by 8 elements;
-    // DCASGD_REPLAY_VECS=1 selects the one-vector kernel for experiments
-    s->replay_vecs = 2;
-    if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) s->replay_vecs = std::atoi(v) == 1 ? 1 : 2;
+    // Two vectors per thread (3 CTAs/SM, 3-stage ring) measured 4-6 % faster on B200 than one vector
+    // per thread (4 CTAs/SM, 5-stage ring) once the vector is long enough to fill the GPU with
+    // the larger CTAs (the per-push control work is shared by 8 elements); short vectors keep one
+    // vector per thread for the parallelism.  DCASGD_REPLAY_VECS=1|2 overrides the choice.
+    int sms = 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
+    s->replay_vecs = blocks_for(c.n, 2) >= 2u * (unsigned)sms ? 2 : 1;
+    if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) { const int k = std::atoi(v); if (k == 1 || k == 2) s->replay_vecs = k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
