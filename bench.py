@@ -50,7 +50,7 @@ FALLBACK_HBM_GBS = 6650.0
 # of the benchmark by its algorithmic bytes.  Tied to the kernel sources by hash: a changed kernel
 # voids the figure (reported as null).  Summary: profiles/k_replay_adaptive_f32_c3_window32.md
 NCU_TRAFFIC: dict[str, dict] = {
-    "k_replay<adaptive,f32>": {"src": "86b9db7894499065", "dram_bytes_per_algorithmic_byte": 0.9895},
+    "k_replay<adaptive,f32>": {"src": "47a321aa58c88c2c", "dram_bytes_per_algorithmic_byte": 0.9895},
 }
 
 
