@@ -50,7 +50,7 @@ FALLBACK_HBM_GBS = 6650.0
 # of the benchmark by its algorithmic bytes.  Tied to the kernel sources by hash: a changed kernel
 # voids the figure (reported as null).  Summary: profiles/k_replay_adaptive_f32_c3_window32.md
 NCU_TRAFFIC: dict[str, dict] = {
-    "k_replay<adaptive,f32>": {"src": "47a321aa58c88c2c", "dram_bytes_per_algorithmic_byte": 0.9895},
+    "k_replay<adaptive,f32>": {"src": "9c0d09226ebf9c0c", "dram_bytes_per_algorithmic_byte": 0.9895},
 }
 
 
@@ -340,7 +340,10 @@ def run_b200(args) -> None:
     max_ms, tot_units = acct.aggregate_over_ranks(total_ms, units * K, dist if world > 1 else None)
     value = tot_units / (max_ms * 1e-3)
 
-    progs = B.plan_log(ev, wl.M, args.window_k, wl.eta)
+    h = create()
+    slot_cap = B.dcasgd_get_window_slot_cap(h)       # cut the log exactly as dcasgd_apply_log does
+    B.dcasgd_destroy(h)
+    progs = B.plan_log(ev, wl.M, args.window_k, wl.eta, slot_cap)
     win_launches = sum(1 for p in progs if acct.window_bytes(p, wl.adaptive, wl.bf16_grad))
     win_bytes = sum(acct.window_bytes(p, wl.adaptive, wl.bf16_grad) for p in progs) * wl.n
     peak, peak_kind = hbm_peak()
@@ -370,7 +373,7 @@ def run_b200(args) -> None:
             if wk == 1:
                 b = acct.unfused_log_bytes(n_push, n_pull, wl.adaptive, wl.bf16_grad) * wl.n
             else:
-                b = sum(acct.window_bytes(p, wl.adaptive, wl.bf16_grad) for p in B.plan_log(ev, wl.M, wk, wl.eta)) * wl.n
+                b = sum(acct.window_bytes(p, wl.adaptive, wl.bf16_grad) for p in B.plan_log(ev, wl.M, wk, wl.eta, slot_cap)) * wl.n
             variants[name] = {"value": units * K / (t_ms * 1e-3), "unit": UNIT, "ms_per_step": t_ms / K,
                               "launches_per_step": ps, "achieved_gbs": b * K / (r_ms * 1e-3) / 1e9,
                               "frac": b * K / (r_ms * 1e-3) / 1e9 / peak, "bytes_per_element_per_push": b / units}

@@ -162,7 +162,7 @@ int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, voi
  *                     comes after step j; w is written to their w_bak slab.  Pulls that are
  *                     superseded inside the window without being used cost nothing.
  * The window is shortened (n_records < window_k) when it would need more than
- * DCASGD_MAX_WINDOW_SLOTS live snapshots, DCASGD_MAX_WINDOW_PUSHES pushes or
+ * max_slots (at most DCASGD_MAX_WINDOW_SLOTS) live snapshots, DCASGD_MAX_WINDOW_PUSHES pushes or
  * DCASGD_MAX_WINDOW_STORES stores; the remaining records start the next window. */
 #define DCASGD_MAX_WINDOW_PUSHES 128
 #define DCASGD_MAX_WINDOW_STORES 192
@@ -184,9 +184,15 @@ typedef struct {
 } dcasgd_window_program;
 
 /* Compiles the window that starts at ev[0] (host, count records available, at most window_k
- * taken).  Records must be valid (kind, worker < num_workers); DCASGD_ELOG otherwise. */
+ * taken), using at most max_slots in-window snapshot slots (0 = DCASGD_MAX_WINDOW_SLOTS).
+ * Records must be valid (kind, worker < num_workers); DCASGD_ELOG otherwise. */
 int dcasgd_compile_window(const dcasgd_event *ev, uint64_t count, uint32_t num_workers, uint32_t window_k,
-                          float default_eta, dcasgd_window_program *out);
+                          float default_eta, uint32_t max_slots, dcasgd_window_program *out);
+
+/* The slot limit dcasgd_apply_log passes to the compiler for this server (it keeps the shared
+ * memory of a window small enough for two or more CTAs per SM): with it,
+ * dcasgd_compile_window cuts a log exactly as dcasgd_apply_log does. */
+int dcasgd_get_window_slot_cap(const dcasgd_server *s, uint32_t *max_slots);
 
 #ifdef __cplusplus
 }

@@ -30,7 +30,8 @@ MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
 # every symbol include/dcasgd.h declares
 SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
            "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_last_error",
-           "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window", "dcasgd_check_adaptive_lambda"]
+           "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window", "dcasgd_check_adaptive_lambda",
+           "dcasgd_get_window_slot_cap"]
 
 
 class Config(C.Structure):
@@ -76,7 +77,9 @@ def lib() -> C.CDLL:
         L.dcasgd_get_step.argtypes = [vp, C.POINTER(u64)]
         L.dcasgd_set_step.argtypes = [vp, u64]
         L.dcasgd_get_launch_count.argtypes = [vp, C.POINTER(u64)]
-        L.dcasgd_compile_window.argtypes = [vp, u64, u32, u32, C.c_float, C.POINTER(WindowProgram)]
+        L.dcasgd_compile_window.argtypes = [vp, u64, u32, u32, C.c_float, u32, C.POINTER(WindowProgram)]
+        L.dcasgd_get_window_slot_cap.argtypes = [vp, C.POINTER(u32)]
+        L.dcasgd_get_window_slot_cap.restype = C.c_int
         L.dcasgd_check_adaptive_lambda.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp]
         L.dcasgd_check_adaptive_lambda.restype = C.c_int
         for name in ("dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
@@ -165,13 +168,19 @@ def dcasgd_version() -> int:
     return int(lib().dcasgd_version())
 
 
-def dcasgd_compile_window(ev, num_workers, window_k, default_eta=0.0) -> WindowProgram:
+def dcasgd_compile_window(ev, num_workers, window_k, default_eta=0.0, max_slots=0) -> WindowProgram:
     """Host only (no GPU needed): the step program of the window that starts at ev[0]."""
     ev = np.ascontiguousarray(ev)
     out = WindowProgram()
     _check(lib().dcasgd_compile_window(ev.ctypes.data if ev.size else None, ev.size, num_workers, window_k,
-                                       default_eta, C.byref(out)))
+                                       default_eta, max_slots, C.byref(out)))
     return out
+
+
+def dcasgd_get_window_slot_cap(h) -> int:
+    cap = C.c_uint32()
+    _check(lib().dcasgd_get_window_slot_cap(h, C.byref(cap)))
+    return cap.value
 
 
 def dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, mismatches_dev, stream=None) -> None:
@@ -180,11 +189,12 @@ def dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, mismatches_dev, strea
     _check(lib().dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, stream, _ptr(mismatches_dev)))
 
 
-def plan_log(ev, num_workers, window_k, default_eta=0.0) -> list[WindowProgram]:
-    """All windows of a log, as dcasgd_apply_log would cut them."""
+def plan_log(ev, num_workers, window_k, default_eta=0.0, max_slots=0) -> list[WindowProgram]:
+    """All windows of a log, as dcasgd_apply_log cuts them when max_slots is the server's
+    dcasgd_get_window_slot_cap."""
     out, r = [], 0
     while r < len(ev):
-        p = dcasgd_compile_window(ev[r:], num_workers, window_k, default_eta)
+        p = dcasgd_compile_window(ev[r:], num_workers, window_k, default_eta, max_slots)
         out.append(p)
         r += p.n_records
     return out

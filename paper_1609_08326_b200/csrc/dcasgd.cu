@@ -19,6 +19,7 @@ struct dcasgd_server {
     cudaStream_t stream;
     int device;
     int replay_vecs;     // 16-byte vectors per thread in the fused replay kernel (1 or 2)
+    uint32_t slot_cap;   // in-window snapshot slots a window may use (keeps >= 2 CTAs per SM resident)
     uint64_t t;          // pushes applied (Algorithm 2's t)
     uint64_t launches;   // kernels launched through this handle
 };
@@ -276,6 +277,11 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
     s->replay_vecs = blocks_for(c.n, 2) >= 2u * (unsigned)sms ? 2 : 1;
     if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) { const int k = std::atoi(v); if (k == 1 || k == 2) s->replay_vecs = k; }
+    // A slot costs 4 KB (8 KB with two vectors per thread) of shared memory per CTA on top of the
+    // staging ring.  Long windows over many workers would take all 16 slots and leave one CTA
+    // per SM; capping the slots cuts such a window a little earlier and keeps two or more resident.
+    s->slot_cap = 8;
+    if (const char* v = std::getenv("DCASGD_WINDOW_SLOTS")) { const int k = std::atoi(v); if (k >= 1 && k <= DCASGD_MAX_WINDOW_SLOTS) s->slot_cap = (uint32_t)k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
@@ -351,7 +357,7 @@ int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, c
         dcasgd_window_program wp;
         uint64_t r = 0;
         while (r < count) {
-            if ((rc = wc.compile(ev + r, count - r, window_k, c.eta, &wp))) return rc;
+            if ((rc = wc.compile(ev + r, count - r, window_k, c.eta, s->slot_cap, &wp))) return rc;
             if ((rc = launch_window(s, wp, grad_pool, grad_stride_bytes))) return rc;
             r += wp.n_records;
         }
@@ -391,6 +397,12 @@ int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, voi
         lambda0, b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("lambda self-check kernel", e);
+    return DCASGD_OK;
+}
+
+int dcasgd_get_window_slot_cap(const dcasgd_server* s, uint32_t* max_slots) {
+    if (!s || !max_slots) return fail(DCASGD_EINVAL, "dcasgd_get_window_slot_cap: NULL argument");
+    *max_slots = s->slot_cap;
     return DCASGD_OK;
 }
 

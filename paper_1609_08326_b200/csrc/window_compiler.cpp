@@ -33,7 +33,7 @@ namespace {
 // One attempt at compiling records [0,K).  Returns 0 on success, otherwise the smaller K (>= 1)
 // at which the window has to end.
 uint64_t attempt(WindowCompiler& c, const dcasgd_event* ev, uint64_t K, float default_eta,
-                 dcasgd_window_program* out) {
+                 int32_t max_slots, dcasgd_window_program* out) {
     auto &uses = c.uses, &pending = c.pending, &remaining = c.remaining;
     auto &is_last = c.is_last, &seen = c.seen, &pulled = c.pulled;
     auto &first_consumer = c.first_consumer, &first_push = c.first_push;
@@ -91,7 +91,7 @@ uint64_t attempt(WindowCompiler& c, const dcasgd_event* ev, uint64_t K, float de
             if (uses[r] > 0) {
                 int32_t s = out->save_slot[j];
                 if (s < 0) {
-                    for (int32_t k = 0; k < DCASGD_MAX_WINDOW_SLOTS; ++k)
+                    for (int32_t k = 0; k < max_slots; ++k)
                         if (slot_ref[k] == 0) { s = k; break; }
                     if (s < 0) { cut = first_consumer[r]; break; }   // no slot: end before its first use
                     out->save_slot[j] = s;
@@ -123,7 +123,8 @@ WindowCompiler::WindowCompiler(uint32_t num_workers)
       pulled(num_workers, 0), first_push(num_workers, 0), cur_slot(num_workers, -1) {}
 
 int WindowCompiler::compile(const dcasgd_event* ev, uint64_t count, uint32_t window_k, float default_eta,
-                            dcasgd_window_program* out) {
+                            uint32_t max_slots, dcasgd_window_program* out) {
+    if (max_slots == 0 || max_slots > DCASGD_MAX_WINDOW_SLOTS) max_slots = DCASGD_MAX_WINDOW_SLOTS;
     uint64_t K = count < window_k ? count : window_k;
     for (uint64_t r = 0; r < K; ++r) {
         if (ev[r].kind > DCASGD_PUSH) { set_error("log record %llu: unknown kind %u", (unsigned long long)r, ev[r].kind); return DCASGD_ELOG; }
@@ -132,7 +133,7 @@ int WindowCompiler::compile(const dcasgd_event* ev, uint64_t count, uint32_t win
     }
     if (uses.size() < K) { uses.resize(K); is_last.resize(K); first_consumer.resize(K); }
     for (;;) {
-        uint64_t cut = attempt(*this, ev, K, default_eta, out);
+        uint64_t cut = attempt(*this, ev, K, default_eta, (int32_t)max_slots, out);
         if (cut == 0) return DCASGD_OK;
         K = cut;
     }
@@ -141,16 +142,21 @@ int WindowCompiler::compile(const dcasgd_event* ev, uint64_t count, uint32_t win
 }  // namespace dcasgd
 
 extern "C" int dcasgd_compile_window(const dcasgd_event* ev, uint64_t count, uint32_t num_workers,
-                                     uint32_t window_k, float default_eta, dcasgd_window_program* out) {
+                                     uint32_t window_k, float default_eta, uint32_t max_slots,
+                                     dcasgd_window_program* out) {
     using namespace dcasgd;
     if (!ev || !out) { set_error("dcasgd_compile_window: NULL argument"); return DCASGD_EINVAL; }
     if (count == 0 || window_k == 0 || num_workers == 0) {
         set_error("dcasgd_compile_window: count, window_k and num_workers must be positive");
         return DCASGD_EINVAL;
     }
+    if (max_slots > DCASGD_MAX_WINDOW_SLOTS) {
+        set_error("dcasgd_compile_window: max_slots %u > %u", max_slots, (unsigned)DCASGD_MAX_WINDOW_SLOTS);
+        return DCASGD_EINVAL;
+    }
     try {
         WindowCompiler c(num_workers);
-        return c.compile(ev, count, window_k, default_eta, out);
+        return c.compile(ev, count, window_k, default_eta, max_slots, out);
     } catch (...) {
         set_error("dcasgd_compile_window: out of host memory");
         return DCASGD_ENOMEM;

@@ -15,9 +15,10 @@ const char* get_error();
 // Reusable scratch for compiling many windows of one log (per-worker arrays are allocated once).
 struct WindowCompiler {
     explicit WindowCompiler(uint32_t num_workers);
-    // Same contract as dcasgd_compile_window; arguments must be non-NULL and positive.
+    // Same contract as dcasgd_compile_window; arguments must be non-NULL and positive
+    // (max_slots 0 or out of range means DCASGD_MAX_WINDOW_SLOTS).
     int compile(const dcasgd_event* ev, uint64_t count, uint32_t window_k, float default_eta,
-                dcasgd_window_program* out);
+                uint32_t max_slots, dcasgd_window_program* out);
 
     uint32_t M;
     std::vector<uint32_t> uses, pending, remaining;

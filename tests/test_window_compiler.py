@@ -51,11 +51,11 @@ def serial(ev, w0, M, adaptive, eta, lam, mu, eps, grads):
     return s
 
 
-def check(ev, M, K, adaptive=True, n=9, G=5, seed=0, eta=0.1):
+def check(ev, M, K, adaptive=True, n=9, G=5, seed=0, eta=0.1, max_slots=0):
     w0 = synth.normal(n, seed, synth.STREAM_W0, 0.05)
     grads = np.stack([synth.normal(n, seed, synth.STREAM_GRAD0 + k, 0.01) for k in range(G)])
     lam, mu, eps = (2.0, 0.95, 1e-7) if adaptive else (0.04, 0.0, 0.0)
-    progs = B.plan_log(ev, M, K, eta)
+    progs = B.plan_log(ev, M, K, eta, max_slots)
     assert sum(p.n_records for p in progs) == len(ev)
     assert sum(p.n_pushes for p in progs) == int(np.sum(ev["kind"] == PUSH))
     w, wb, ms = interpret(progs, w0, M, adaptive, lam, mu, eps, grads)
@@ -149,3 +149,17 @@ def test_compile_rejects_bad_records():
     with pytest.raises(B.DcasgdError) as e:
         B.dcasgd_compile_window(synth.make_log([]), 4, 8, 0.1)
     assert e.value.status == B.EINVAL
+
+
+@pytest.mark.parametrize("cap", [1, 2, 3, 8, 16])
+def test_slot_cap_cuts_windows_but_not_results(cap):
+    """A smaller slot budget ends windows earlier; the replay stays the checker's, bit for bit."""
+    ev = synth.event_log(16, 400, synth.ORDER_UNIFORM, synth.PROTO_ASYNC, 5, 0.1, seed=cap)
+    progs = check(ev, 16, 256, max_slots=cap)
+    assert max(p.n_slots for p in progs) <= cap
+    full = B.plan_log(ev, 16, 256, 0.1)
+    assert len(progs) >= len(full)
+    if cap == 16:
+        assert [p.n_records for p in progs] == [p.n_records for p in full]
+    with pytest.raises(B.DcasgdError):
+        B.dcasgd_compile_window(ev, 16, 8, 0.1, max_slots=17)
