@@ -180,7 +180,7 @@ def sample_log(ev, pushes: int):
     return ev[: idx[pushes - 1] + 2] if idx[pushes - 1] + 2 <= len(ev) else ev[: idx[pushes - 1] + 1]
 
 
-def cpu_baseline(wl, ev, w0_np, pool_np, target_s: float = 15.0) -> dict:
+def cpu_baseline(wl, ev, w0_np, pool_np, target_s: float = 30.0) -> dict:
     cores = os.cpu_count() or 1
     probe = sample_log(ev, 8)
     p_probe = int(np.sum(probe["kind"] == synth.PUSH))
