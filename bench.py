@@ -131,6 +131,10 @@ def select_workload(args) -> synth.Workload:
         kw["pushes"] = args.pushes
     if args.pool:
         kw["num_grads"] = args.pool
+    if args.n:
+        kw["n"] = args.n
+    if args.workers:
+        kw["M"] = args.workers
     return wl.scaled(**kw) if kw else wl
 
 
@@ -436,6 +440,8 @@ def main() -> None:
     ap.add_argument("--window-k", type=int, default=32)
     ap.add_argument("--pushes", type=int, default=0, help="shorten the log (profiling runs)")
     ap.add_argument("--pool", type=int, default=0, help="shrink the gradient pool (profiling runs)")
+    ap.add_argument("--n", type=int, default=0, help="override the parameter count (profiling runs)")
+    ap.add_argument("--workers", type=int, default=0, help="override the worker count (profiling runs)")
     ap.add_argument("--ref-pushes", type=int, default=24, help="pushes per step of the reference arm")
     ap.add_argument("--headline-only", action="store_true", help="skip variants, single kernels, e2e, CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
