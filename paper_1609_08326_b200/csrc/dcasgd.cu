@@ -88,7 +88,7 @@ int after_launch(dcasgd_server* s, const char* what) {
 int launch_pull(dcasgd_server* s, uint32_t m, float* out_w) {
     const dcasgd_config& c = s->cfg;
     if (c.n == 0) return DCASGD_OK;
-    k_pull<<<blocks_for(c.n, kPushUnroll), kThreads, 0, s->stream>>>(
+    k_pull<<<blocks_for(c.n, kPullUnroll), kThreads, 0, s->stream>>>(
         c.w, c.w_bak + (uint64_t)m * c.w_bak_stride, out_w, c.n);
     return after_launch(s, "pull kernel");
 }
