@@ -16,10 +16,15 @@
  *              constant variant (DC-ASGD-c): lambda_t = lambda
  *              adaptive variant (DC-ASGD-a): ms <- mu*ms + (1-mu)*g.g ;  lambda_t = lambda / sqrt(ms + eps)
  *
+ *   momentum   (optional; Section 6 mentions momentum variants in a footnote and prints no formula.
+ *              Reading: classical momentum on the delay-compensated gradient u = g + lambda_t*g.g.(w - w_bak[m]):
+ *              v <- beta*v + eta*u ;  w <- w - v ;  v starts at 0; beta = 0 is Eq. 10 itself)
+ *
  * Arithmetic: IEEE binary32, every operation rounded to nearest on its own (no fused
  * multiply-add), in this order per element:
  *     gg = g*g ; [ms = mu*ms + (1-mu)*gg ; lam = lambda / sqrt(ms + eps)] ;
  *     d = w - w_bak[m] ; c = (lam*gg)*d ; u = g + c ; w = w - eta*u
+ *     (momentum: p = eta*u ; v = beta*v + p ; w = w - v)
  * with (1-mu) rounded once on the host.  bfloat16 gradients are widened exactly first.  Results
  * therefore do not depend on which kernel (single push or fused window) applied an event.
  *
@@ -86,6 +91,9 @@ typedef struct {
   uint64_t w_bak_stride; /* floats between slabs: >= n and a multiple of 4 */
   float *ms;             /* device, n floats, 16-byte aligned; NULL if and only if DCASGD_CONST */
   void *stream;          /* cudaStream_t; NULL is the legacy default stream */
+  float *v;              /* device, n floats, 16-byte aligned: velocity of the momentum variant; NULL = no momentum */
+  float beta;            /* momentum coefficient in [0,1); must be 0 when v is NULL */
+  uint32_t reserved;     /* 0 */
 } dcasgd_config;
 
 /* One record of the server's message log, 16 bytes. */
@@ -97,8 +105,8 @@ typedef struct {
   float eta;        /* PUSH: learning rate of this update, < 0 = the server's default; PULL: ignored */
 } dcasgd_event;
 
-/* Algorithm 2, "Initialize": t = 0, w_bak[m] = w for every m, ms = 0 (skipped with DCASGD_RESUME).
- * cfg (host) is copied.  *out receives the handle.  w, w_bak, ms must not overlap. */
+/* Algorithm 2, "Initialize": t = 0, w_bak[m] = w for every m, ms = 0, v = 0 (skipped with
+ * DCASGD_RESUME).  cfg (host) is copied.  *out receives the handle.  w, w_bak, ms, v must not overlap. */
 int dcasgd_create(const dcasgd_config *cfg, dcasgd_server **out);
 
 /* Algorithm 2, pull branch: w_bak[m] <- w.  If out_w (device, n floats, 16-byte aligned, not

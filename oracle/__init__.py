@@ -37,13 +37,13 @@ def _bind(path: str) -> C.CDLL:
         getattr(L, f"oracle_init_{suf}").restype = None
         getattr(L, f"oracle_pull_{suf}").argtypes = [u64, u32, vp, vp]
         getattr(L, f"oracle_pull_{suf}").restype = None
-    L.oracle_push_f32.argtypes = [u64, u32, i32] + [C.c_float] * 4 + [vp, vp, vp, vp, i32]
+    L.oracle_push_f32.argtypes = [u64, u32, i32] + [C.c_float] * 4 + [vp, vp, vp, vp, i32, C.c_float, vp]
     L.oracle_push_f32.restype = None
-    L.oracle_push_f64.argtypes = [u64, u32, i32] + [C.c_double] * 4 + [vp, vp, vp, vp]
+    L.oracle_push_f64.argtypes = [u64, u32, i32] + [C.c_double] * 4 + [vp, vp, vp, vp, C.c_double, vp]
     L.oracle_push_f64.restype = None
-    L.oracle_replay_f32.argtypes = [u64, u32, i32] + [C.c_float] * 4 + [vp, vp, vp, vp, u64, vp, u64, u32, i32, vp]
+    L.oracle_replay_f32.argtypes = [u64, u32, i32] + [C.c_float] * 4 + [vp, vp, vp, vp, u64, vp, u64, u32, i32, vp, C.c_float, vp]
     L.oracle_replay_f32.restype = i32
-    L.oracle_replay_f64.argtypes = [u64, u32, i32] + [C.c_double] * 4 + [vp, vp, vp, vp, u64, vp, u64, u32, vp]
+    L.oracle_replay_f64.argtypes = [u64, u32, i32] + [C.c_double] * 4 + [vp, vp, vp, vp, u64, vp, u64, u32, vp, C.c_double, vp]
     L.oracle_replay_f64.restype = i32
     return L
 
@@ -70,7 +70,7 @@ class Server:
     """
 
     def __init__(self, w0, M: int, adaptive: bool, eta: float, lam: float, mu: float = 0.0,
-                 eps: float = 0.0, dtype=np.float32, library: C.CDLL | None = None):
+                 eps: float = 0.0, dtype=np.float32, library: C.CDLL | None = None, beta: float | None = None):
         self.L = library or lib()
         self.dtype = np.dtype(dtype)
         self.suf = "f32" if self.dtype == np.float32 else "f64"
@@ -81,6 +81,8 @@ class Server:
         self.w = np.array(w0, dtype=self.dtype).reshape(-1).copy()
         self.w_bak = np.empty((self.M, self.n), dtype=self.dtype)
         self.ms = np.empty(self.n, dtype=self.dtype) if adaptive else None
+        self.beta = 0.0 if beta is None else beta               # momentum: None = off (no velocity vector)
+        self.v = None if beta is None else np.zeros(self.n, dtype=self.dtype)
         self.t = C.c_uint64(0)
         getattr(self.L, f"oracle_init_{self.suf}")(self.n, self.M, _ptr(self.w), _ptr(self.w_bak),
                                                    _ptr(self.ms))
@@ -100,11 +102,11 @@ class Server:
             assert g.dtype in (np.float32, np.uint16)
             self.L.oracle_push_f32(self.n, m, int(self.adaptive), e, self.lam, self.mu, self.eps,
                                    _ptr(self.w), _ptr(self.w_bak), _ptr(self.ms), _ptr(g),
-                                   int(g.dtype == np.uint16))
+                                   int(g.dtype == np.uint16), self.beta, _ptr(self.v))
         else:
             assert g.dtype == np.float64
             self.L.oracle_push_f64(self.n, m, int(self.adaptive), e, self.lam, self.mu, self.eps,
-                                   _ptr(self.w), _ptr(self.w_bak), _ptr(self.ms), _ptr(g))
+                                   _ptr(self.w), _ptr(self.w_bak), _ptr(self.ms), _ptr(g), self.beta, _ptr(self.v))
         self.t.value += 1
 
     def replay(self, ev: np.ndarray, grads: np.ndarray) -> None:
@@ -120,12 +122,12 @@ class Server:
             rc = self.L.oracle_replay_f32(self.n, self.M, int(self.adaptive), self.eta, self.lam,
                                           self.mu, self.eps, _ptr(self.w), _ptr(self.w_bak),
                                           _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), stride, G,
-                                          int(grads.dtype == np.uint16), C.addressof(self.t))
+                                          int(grads.dtype == np.uint16), C.addressof(self.t), self.beta, _ptr(self.v))
         else:
             assert grads.dtype == np.float64
             rc = self.L.oracle_replay_f64(self.n, self.M, int(self.adaptive), self.eta, self.lam,
                                           self.mu, self.eps, _ptr(self.w), _ptr(self.w_bak),
                                           _ptr(self.ms), _ptr(ev), ev.size, _ptr(grads), stride, G,
-                                          C.addressof(self.t))
+                                          C.addressof(self.t), self.beta, _ptr(self.v))
         if rc != 0:
             raise ValueError(f"oracle rejected the log (code {rc})")

@@ -29,12 +29,21 @@
 //   * A push with no earlier pull uses whatever w_bak(m) holds (w_0 after Initialize).
 //   * bfloat16 gradients widen exactly (16 zero bits appended) before any arithmetic.
 //
+//   * Momentum (optional).  Section 6 says in a footnote that momentum variants were implemented
+//     and gives no formula.  Reading taken: classical (heavy-ball) momentum on the
+//     delay-compensated gradient u, as in the solvers the paper's ResNet code uses:
+//         v = beta*v + eta*u ;  w = w - v          (v starts at 0; beta = 0 is Eq. 10 itself)
+//     with beta*v and eta*u rounded separately, then their sum, then the difference.
+//
 // Pins (tests/test_oracle_pins.py): hand-worked dyadic examples checked against exact rational
 // arithmetic, the closed form of repeated pushes on one snapshot, lambda = 0 against an
 // independent ASGD loop, tau = 0 against plain SGD, MeanSquare against its unrolled sum,
 // mu = 0 against g^2, and a brute-force element-outer replay on tiny inputs.
-// Parity unpinned: nothing in this file.  (The paper's accuracy tables need CIFAR-10/ImageNet
-// and are outside what this checker computes.)
+// Also pinned for momentum: beta = 0 equals the plain update bit for bit; with lambda = 0 and no
+// delay it is textbook momentum SGD; exact rational replay with dyadic beta.
+// Parity unpinned: the CHOICE of the momentum formula (the paper prints none); everything else
+// in this file is pinned.  (The paper's accuracy tables need CIFAR-10/ImageNet and are outside
+// what this checker computes.)
 
 #include <cmath>
 #include <cstdint>
@@ -78,7 +87,7 @@ void pull(uint64_t n, uint32_t m, const T* w, T* wb) {
 // G is the stored gradient type (T, or uint16_t holding bfloat16 when T is float).
 template <class T, class G>
 void push(uint64_t n, uint32_t m, int adaptive, T eta, T lambda, T mu, T eps,
-          T* w, const T* wb, T* ms, const G* g) {
+          T* w, const T* wb, T* ms, const G* g, T beta, T* vel) {
     const T omm = (T)1 - mu;
     const T* snap = wb + (uint64_t)m * n;
     for (uint64_t i = 0; i < n; ++i) {
@@ -100,6 +109,12 @@ void push(uint64_t n, uint32_t m, int adaptive, T eta, T lambda, T mu, T eps,
         c = c * d;
         T u = gi + c;
         T p = eta * u;
+        if (vel) {                                // momentum reading: v = beta*v + eta*u ; w = w - v
+            T bv = beta * vel[i];
+            T nv = bv + p;
+            vel[i] = nv;
+            p = nv;
+        }
         w[i] = w[i] - p;
     }
 }
@@ -107,7 +122,7 @@ void push(uint64_t n, uint32_t m, int adaptive, T eta, T lambda, T mu, T eps,
 template <class T, class G>
 int replay(uint64_t n, uint32_t M, int adaptive, T default_eta, T lambda, T mu, T eps,
            T* w, T* wb, T* ms, const oracle_event* ev, uint64_t count,
-           const G* grads, uint64_t grad_stride, uint32_t num_grads, uint64_t* t) {
+           const G* grads, uint64_t grad_stride, uint32_t num_grads, uint64_t* t, T beta, T* vel) {
     for (uint64_t e = 0; e < count; ++e) {
         const oracle_event& r = ev[e];
         if (r.worker >= M) return ORACLE_BAD_WORKER;
@@ -117,7 +132,7 @@ int replay(uint64_t n, uint32_t M, int adaptive, T default_eta, T lambda, T mu, 
             if (r.grad_id >= num_grads) return ORACLE_BAD_GRAD;
             T eta = r.eta < 0.0f ? default_eta : (T)r.eta;
             push<T, G>(n, r.worker, adaptive, eta, lambda, mu, eps, w, wb, ms,
-                       grads + (uint64_t)r.grad_id * grad_stride);
+                       grads + (uint64_t)r.grad_id * grad_stride, beta, vel);
             if (t) *t += 1;                       // Algorithm 2: t advances on a gradient only
         } else {
             return ORACLE_BAD_KIND;
@@ -136,14 +151,16 @@ void oracle_init_f64(uint64_t n, uint32_t M, const double* w, double* wb, double
 void oracle_pull_f32(uint64_t n, uint32_t m, const float* w, float* wb) { pull<float>(n, m, w, wb); }
 void oracle_pull_f64(uint64_t n, uint32_t m, const double* w, double* wb) { pull<double>(n, m, w, wb); }
 
+// beta, vel: momentum coefficient and velocity vector (n elements, starts at 0); vel == NULL
+// means no momentum.
 void oracle_push_f32(uint64_t n, uint32_t m, int adaptive, float eta, float lambda, float mu, float eps,
-                     float* w, const float* wb, float* ms, const void* g, int g_is_bf16) {
-    if (g_is_bf16) push<float, uint16_t>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, (const uint16_t*)g);
-    else           push<float, float>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, (const float*)g);
+                     float* w, const float* wb, float* ms, const void* g, int g_is_bf16, float beta, float* vel) {
+    if (g_is_bf16) push<float, uint16_t>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, (const uint16_t*)g, beta, vel);
+    else           push<float, float>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, (const float*)g, beta, vel);
 }
 void oracle_push_f64(uint64_t n, uint32_t m, int adaptive, double eta, double lambda, double mu, double eps,
-                     double* w, const double* wb, double* ms, const double* g) {
-    push<double, double>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, g);
+                     double* w, const double* wb, double* ms, const double* g, double beta, double* vel) {
+    push<double, double>(n, m, adaptive, eta, lambda, mu, eps, w, wb, ms, g, beta, vel);
 }
 
 // Serial replay of a log (the repeat-loop of Algorithm 2).  grads: num_grads buffers,
@@ -151,18 +168,19 @@ void oracle_push_f64(uint64_t n, uint32_t m, int adaptive, double eta, double la
 int oracle_replay_f32(uint64_t n, uint32_t M, int adaptive, float default_eta, float lambda, float mu,
                       float eps, float* w, float* wb, float* ms, const oracle_event* ev, uint64_t count,
                       const void* grads, uint64_t grad_stride, uint32_t num_grads, int g_is_bf16,
-                      uint64_t* t) {
+                      uint64_t* t, float beta, float* vel) {
     if (g_is_bf16)
         return replay<float, uint16_t>(n, M, adaptive, default_eta, lambda, mu, eps, w, wb, ms, ev, count,
-                                       (const uint16_t*)grads, grad_stride, num_grads, t);
+                                       (const uint16_t*)grads, grad_stride, num_grads, t, beta, vel);
     return replay<float, float>(n, M, adaptive, default_eta, lambda, mu, eps, w, wb, ms, ev, count,
-                                (const float*)grads, grad_stride, num_grads, t);
+                                (const float*)grads, grad_stride, num_grads, t, beta, vel);
 }
 int oracle_replay_f64(uint64_t n, uint32_t M, int adaptive, double default_eta, double lambda, double mu,
                       double eps, double* w, double* wb, double* ms, const oracle_event* ev, uint64_t count,
-                      const double* grads, uint64_t grad_stride, uint32_t num_grads, uint64_t* t) {
+                      const double* grads, uint64_t grad_stride, uint32_t num_grads, uint64_t* t,
+                      double beta, double* vel) {
     return replay<double, double>(n, M, adaptive, default_eta, lambda, mu, eps, w, wb, ms, ev, count,
-                                  grads, grad_stride, num_grads, t);
+                                  grads, grad_stride, num_grads, t, beta, vel);
 }
 
 }  // extern "C"

@@ -5,6 +5,7 @@ Per element, fp32 state:
     pull                      8            read w, write w_bak[m]
     push, constant lambda    12 + g        w in and out, w_bak[m] in, gradient in (g = 4 fp32, 2 bf16)
     push, adaptive           20 + g        + MeanSquare in and out
+    (momentum variant: + 8 per push, or per window, for the velocity in and out)
     fused window              S + g*P + 4*R + 4*W
         S = 8 (constant) or 16 (adaptive): w (and ms) in and out once per window
         P = pushes in the window, R = pushes that read a pre-window backup,
@@ -21,19 +22,20 @@ def pull_bytes() -> int:
     return 8
 
 
-def push_bytes(adaptive: bool, bf16: bool) -> int:
-    return (20 if adaptive else 12) + grad_bytes(bf16)
+def push_bytes(adaptive: bool, bf16: bool, momentum: bool = False) -> int:
+    return (20 if adaptive else 12) + grad_bytes(bf16) + (8 if momentum else 0)
 
 
 def init_bytes(M: int, adaptive: bool) -> int:
     return 4 + 4 * M + (4 if adaptive else 0)
 
 
-def window_bytes(prog, adaptive: bool, bf16: bool) -> int:
+def window_bytes(prog, adaptive: bool, bf16: bool, momentum: bool = False) -> int:
     """Bytes per element of one compiled window (a WindowProgram); 0 if it launches nothing."""
     if prog.n_pushes == 0 and prog.n_stores == 0:
         return 0
-    return (16 if adaptive else 8) + grad_bytes(bf16) * prog.n_pushes + 4 * prog.n_snapshot_reads + 4 * prog.n_stores
+    state = (16 if adaptive else 8) + (8 if momentum else 0)
+    return state + grad_bytes(bf16) * prog.n_pushes + 4 * prog.n_snapshot_reads + 4 * prog.n_stores
 
 
 def unfused_log_bytes(n_pushes: int, n_pulls: int, adaptive: bool, bf16: bool) -> int:

@@ -38,7 +38,8 @@ class Config(C.Structure):
     _fields_ = [("n", C.c_uint64), ("num_workers", C.c_uint32), ("variant", C.c_uint32),
                 ("grad_dtype", C.c_uint32), ("eta", C.c_float), ("lambda_", C.c_float),
                 ("mu", C.c_float), ("eps", C.c_float), ("flags", C.c_uint32), ("w", C.c_void_p), ("w_bak", C.c_void_p),
-                ("w_bak_stride", C.c_uint64), ("ms", C.c_void_p), ("stream", C.c_void_p)]
+                ("w_bak_stride", C.c_uint64), ("ms", C.c_void_p), ("stream", C.c_void_p),
+                ("v", C.c_void_p), ("beta", C.c_float), ("reserved", C.c_uint32)]
 
 
 class WindowProgram(C.Structure):
@@ -120,9 +121,9 @@ def _ptr(x) -> int | None:
 # ---------------------------------------------------------------- the C calls, one to one
 
 def dcasgd_create(n, num_workers, variant, grad_dtype, eta, lam, mu, eps, w, w_bak, w_bak_stride,
-                  ms, stream=None, flags=0) -> int:
+                  ms, stream=None, flags=0, v=None, beta=0.0) -> int:
     cfg = Config(n, num_workers, variant, grad_dtype, eta, lam, mu, eps, flags, _ptr(w), _ptr(w_bak),
-                 w_bak_stride, _ptr(ms), stream)
+                 w_bak_stride, _ptr(ms), stream, _ptr(v), beta, 0)
     h = C.c_void_p()
     _check(lib().dcasgd_create(C.byref(cfg), C.byref(h)))
     return h.value
@@ -255,8 +256,10 @@ class Server:
     """Owns the torch tensors a server borrows (w, w_bak, ms) and the handle."""
 
     def __init__(self, w0, num_workers: int, adaptive: bool, eta: float, lam: float, mu: float = 0.0,
-                 eps: float = 0.0, bf16_grad: bool = False, device="cuda", stream=None, state: dict | None = None):
-        """`state` (from state_dict()) resumes a saved server instead of initialising from w0."""
+                 eps: float = 0.0, bf16_grad: bool = False, device="cuda", stream=None, state: dict | None = None,
+                 beta: float | None = None):
+        """`state` (from state_dict()) resumes a saved server instead of initialising from w0.
+        `beta` (not None) selects the momentum variant with that coefficient."""
         import torch
         self.torch = torch
         self.device = torch.device(device)
@@ -267,17 +270,21 @@ class Server:
         self.w = w0.to(self.device, copy=True).contiguous()
         self.w_bak_buf = torch.empty(self.M * self.stride, dtype=torch.float32, device=self.device)
         self.ms = torch.empty(self.n, dtype=torch.float32, device=self.device) if adaptive else None
+        self.v = torch.empty(self.n, dtype=torch.float32, device=self.device) if beta is not None else None
         if state is not None:
             self.w_bak_buf.view(self.M, self.stride)[:, : self.n].copy_(state["w_bak"])
             if adaptive:
                 self.ms.copy_(state["ms"])
+            if beta is not None:
+                self.v.copy_(state["v"])
         self.bf16_grad = bool(bf16_grad)
         self.stream = stream
         s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(self.device).cuda_stream
         with torch.cuda.device(self.device):
             self.h = dcasgd_create(self.n, self.M, ADAPTIVE if adaptive else CONST, BF16 if bf16_grad else F32,
                                    eta, lam, mu, eps, self.w, self.w_bak_buf, self.stride, self.ms, s,
-                                   flags=RESUME if state is not None else 0)
+                                   flags=RESUME if state is not None else 0, v=self.v,
+                                   beta=0.0 if beta is None else beta)
         if state is not None:
             dcasgd_set_step(self.h, int(state["t"]))
 
@@ -285,7 +292,7 @@ class Server:
         """The whole server state (w, every backup, MeanSquare, t) as host copies: a checkpoint."""
         self.torch.cuda.synchronize(self.device)
         return {"w": self.w.cpu(), "w_bak": self.w_bak.cpu(), "ms": None if self.ms is None else self.ms.cpu(),
-                "t": self.step}
+                "v": None if self.v is None else self.v.cpu(), "t": self.step}
 
     @property
     def w_bak(self):

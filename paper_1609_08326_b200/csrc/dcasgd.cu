@@ -54,17 +54,18 @@ int cuda_fail(const char* what, cudaError_t e) {
 }
 
 // The state arrays of a server as byte ranges, for overlap checks against caller buffers.
-int state_ranges(const dcasgd_config& c, Range out[3]) {
+int state_ranges(const dcasgd_config& c, Range out[4]) {
     int k = 0;
     out[k++] = range_of(c.w, c.n * 4, "w");
     const uint64_t bak = c.n == 0 ? 0 : (uint64_t)c.num_workers * c.w_bak_stride * 4;   // every slab is stride floats long
     out[k++] = range_of(c.w_bak, bak, "w_bak");
     if (c.ms) out[k++] = range_of(c.ms, c.n * 4, "ms");
+    if (c.v) out[k++] = range_of(c.v, c.n * 4, "v");
     return k;
 }
 
 int check_foreign(const dcasgd_config& c, const void* p, uint64_t bytes, const char* name) {
-    Range st[3];
+    Range st[4];
     const int k = state_ranges(c, st);
     const Range r = range_of(p, bytes, name);
     for (int i = 0; i < k; ++i)
@@ -102,15 +103,22 @@ int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
     a.wb_m = c.w_bak + (uint64_t)m * c.w_bak_stride;
     a.ms = c.ms;
     a.g = g;
+    a.vel = c.v;
     a.n = c.n;
     a.eta = eta < 0.0f ? c.eta : eta;
     a.h = s->h;
     const unsigned grid = blocks_for(c.n, kPushUnroll);
-    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
-    if (ad && bf)       k_push<true, true><<<grid, kThreads, 0, s->stream>>>(a);
-    else if (ad)        k_push<true, false><<<grid, kThreads, 0, s->stream>>>(a);
-    else if (bf)        k_push<false, true><<<grid, kThreads, 0, s->stream>>>(a);
-    else                k_push<false, false><<<grid, kThreads, 0, s->stream>>>(a);
+    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
+#define DCASGD_LAUNCH_PUSH(AD, BF)                                                           \
+    do {                                                                                     \
+        if (mom) k_push<AD, BF, true><<<grid, kThreads, 0, s->stream>>>(a);                  \
+        else     k_push<AD, BF, false><<<grid, kThreads, 0, s->stream>>>(a);                 \
+    } while (0)
+    if (ad && bf)       DCASGD_LAUNCH_PUSH(true, true);
+    else if (ad)        DCASGD_LAUNCH_PUSH(true, false);
+    else if (bf)        DCASGD_LAUNCH_PUSH(false, true);
+    else                DCASGD_LAUNCH_PUSH(false, false);
+#undef DCASGD_LAUNCH_PUSH
     return after_launch(s, "push kernel");
 }
 
@@ -141,17 +149,23 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.w = c.w;
     a.w_bak = c.w_bak;
     a.ms = c.ms;
+    a.vel = c.v;
     a.grad_pool = static_cast<const char*>(grad_pool);
     a.n = c.n;
     a.h = s->h;
     const int V = s->replay_vecs;
     const unsigned grid = blocks_for(c.n, V);
     const size_t smem = replay_smem_bytes(wp.n_slots, V);
-    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16;
+    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
 #define DCASGD_LAUNCH_REPLAY(AD, BF)                                                         \
     do {                                                                                     \
-        if (V == 2) k_replay<AD, BF, 2><<<grid, kThreads, smem, s->stream>>>(a, p);          \
-        else        k_replay<AD, BF, 1><<<grid, kThreads, smem, s->stream>>>(a, p);          \
+        if (mom) {                                                                           \
+            if (V == 2) k_replay<AD, BF, true, 2><<<grid, kThreads, smem, s->stream>>>(a, p); \
+            else        k_replay<AD, BF, true, 1><<<grid, kThreads, smem, s->stream>>>(a, p); \
+        } else {                                                                             \
+            if (V == 2) k_replay<AD, BF, false, 2><<<grid, kThreads, smem, s->stream>>>(a, p); \
+            else        k_replay<AD, BF, false, 1><<<grid, kThreads, smem, s->stream>>>(a, p); \
+        }                                                                                    \
     } while (0)
     if (ad && bf)       DCASGD_LAUNCH_REPLAY(true, true);
     else if (ad)        DCASGD_LAUNCH_REPLAY(true, false);
@@ -161,13 +175,18 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     return after_launch(s, "window replay kernel");
 }
 
-template <bool AD, bool BF>
-cudaError_t allow_slots() {
-    cudaError_t e = cudaFuncSetAttribute(k_replay<AD, BF, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <bool AD, bool BF, bool MOM>
+cudaError_t allow_slots_one() {
+    cudaError_t e = cudaFuncSetAttribute(k_replay<AD, BF, MOM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 1));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_replay<AD, BF, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(k_replay<AD, BF, MOM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 2));
+}
+template <bool AD, bool BF>
+cudaError_t allow_slots() {
+    const cudaError_t e = allow_slots_one<AD, BF, false>();
+    return e != cudaSuccess ? e : allow_slots_one<AD, BF, true>();
 }
 
 int check_server(const dcasgd_server* s, const char* fn) {
@@ -219,14 +238,20 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     } else if (c.ms) {
         return fail(DCASGD_EINVAL, "dcasgd_create: ms must be NULL for the constant variant");
     }
+    if (c.reserved != 0) return fail(DCASGD_EINVAL, "dcasgd_create: reserved must be 0");
+    if (c.v) {
+        if (!(c.beta >= 0.0f && c.beta < 1.0f)) return fail(DCASGD_EINVAL, "dcasgd_create: beta must be in [0,1)");
+    } else if (c.beta != 0.0f) {
+        return fail(DCASGD_EINVAL, "dcasgd_create: beta must be 0 without a velocity vector v");
+    }
     if (c.n) {
         if (!c.w || !c.w_bak) return fail(DCASGD_EINVAL, "dcasgd_create: w and w_bak are required");
         if (c.w_bak_stride < c.n) return fail(DCASGD_EINVAL, "dcasgd_create: w_bak_stride < n");
         if (c.w_bak_stride % 4) return fail(DCASGD_EALIGN, "dcasgd_create: w_bak_stride must be a multiple of 4 floats");
-        if (!aligned16(c.w) || !aligned16(c.w_bak) || (c.ms && !aligned16(c.ms)))
-            return fail(DCASGD_EALIGN, "dcasgd_create: w, w_bak and ms must be 16-byte aligned");
+        if (!aligned16(c.w) || !aligned16(c.w_bak) || (c.ms && !aligned16(c.ms)) || (c.v && !aligned16(c.v)))
+            return fail(DCASGD_EALIGN, "dcasgd_create: w, w_bak, ms and v must be 16-byte aligned");
         if (c.n > (uint64_t)1 << 40) return fail(DCASGD_EINVAL, "dcasgd_create: n too large");
-        Range st[3];
+        Range st[4];
         const int k = state_ranges(c, st);
         for (int i = 0; i < k; ++i)
             for (int j = i + 1; j < k; ++j)
@@ -238,9 +263,9 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail("dcasgd_create: cudaGetDevice", e);
     if (c.n) {
-        const void* ptrs[3] = {c.w, c.w_bak, c.ms};
-        const char* names[3] = {"w", "w_bak", "ms"};
-        for (int i = 0; i < 3; ++i) {
+        const void* ptrs[4] = {c.w, c.w_bak, c.ms, c.v};
+        const char* names[4] = {"w", "w_bak", "ms", "v"};
+        for (int i = 0; i < 4; ++i) {
             if (!ptrs[i]) continue;
             cudaPointerAttributes at;
             e = cudaPointerGetAttributes(&at, ptrs[i]);
@@ -262,6 +287,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->h.mu = adaptive ? c.mu : 0.0f;
     s->h.omm = 1.0f - s->h.mu;
     s->h.eps = adaptive ? c.eps : 0.0f;
+    s->h.beta = c.v ? c.beta : 0.0f;
     const float al = std::fabs(c.lambda);
     s->h.fast = (al >= 0x1p-60f && al < 0x1p60f) ? 1u : 0u;
     if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) s->h.fast = 0u; }
@@ -284,7 +310,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     if (const char* v = std::getenv("DCASGD_WINDOW_SLOTS")) { const int k = std::atoi(v); if (k >= 1 && k <= DCASGD_MAX_WINDOW_SLOTS) s->slot_cap = (uint32_t)k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
-        k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.n);
+        k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.v, c.n);
         const int rc = after_launch(s, "init kernel");
         if (rc != DCASGD_OK) { delete s; return rc; }
     }

@@ -30,13 +30,13 @@ def to_device(pool: np.ndarray):
     return torch.from_numpy(pool).cuda()
 
 
-def gpu_server(wl: synth.Workload, w0: np.ndarray, stream=None) -> B.Server:
-    return B.Server(w0, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, wl.bf16_grad, stream=stream)
+def gpu_server(wl: synth.Workload, w0: np.ndarray, stream=None, beta=None) -> B.Server:
+    return B.Server(w0, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, wl.bf16_grad, stream=stream, beta=beta)
 
 
-def cpu_server(wl: synth.Workload, w0: np.ndarray) -> oracle.Server:
+def cpu_server(wl: synth.Workload, w0: np.ndarray, beta=None) -> oracle.Server:
     return oracle.Server(w0, wl.M, wl.adaptive, np.float32(wl.eta), np.float32(wl.lam), np.float32(wl.mu),
-                         np.float32(wl.eps))
+                         np.float32(wl.eps), beta=None if beta is None else np.float32(beta))
 
 
 def sample_indices(n: int, seg_len: int = 0, nseg: int = 1, edge: int = 4096, every: int = 1009) -> np.ndarray:
@@ -58,6 +58,8 @@ def assert_state_equal(gpu: B.Server, cpu: oracle.Server, idx: np.ndarray | None
     pairs = [("w", sel(gpu.w), cpu.w), ("w_bak", sel(gpu.w_bak), cpu.w_bak)]
     if cpu.ms is not None:
         pairs.append(("ms", sel(gpu.ms), cpu.ms))
+    if cpu.v is not None:
+        pairs.append(("v", sel(gpu.v), cpu.v))
     for name, got, want in pairs:
         assert got.shape == want.shape
         # NaN payloads are not fixed by IEEE 754 (x86 and the GPU pick different quiet NaNs)

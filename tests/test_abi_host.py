@@ -33,8 +33,9 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_the_header():
-    assert C.sizeof(B.Config) == 80
+    assert C.sizeof(B.Config) == 96
     assert B.Config.flags.offset == 36 and B.Config.w.offset == 40 and B.Config.w_bak_stride.offset == 56 and B.Config.ms.offset == 64 and B.Config.stream.offset == 72
+    assert B.Config.v.offset == 80 and B.Config.beta.offset == 88 and B.Config.reserved.offset == 92
     assert synth.EVENT_DTYPE.itemsize == 16
     words = 6 + 3 * B.MAX_WINDOW_PUSHES + (B.MAX_WINDOW_PUSHES + 1) + (B.MAX_WINDOW_PUSHES + 2) + B.MAX_WINDOW_STORES
     assert C.sizeof(B.WindowProgram) == 4 * words
@@ -54,6 +55,8 @@ def _create(**kw):
 @pytest.mark.parametrize("kw,status", [
     (dict(num_workers=0), B.EINVAL), (dict(num_workers=70000), B.EINVAL),
     (dict(variant=2), B.EINVAL), (dict(grad_dtype=2), B.EINVAL), (dict(flags=2), B.EINVAL),
+    (dict(beta=0.9), B.EINVAL), (dict(v=0x50000, beta=1.0), B.EINVAL), (dict(v=0x50000, beta=-0.5), B.EINVAL),
+    (dict(v=0x50004, beta=0.9), B.EALIGN), (dict(v=0x10010, beta=0.9), B.EINVAL),       # v inside w
     (dict(eta=float("nan")), B.EINVAL), (dict(lam=float("inf")), B.EINVAL),
     (dict(mu=1.0), B.EINVAL), (dict(mu=-0.1), B.EINVAL), (dict(eps=-1e-7), B.EINVAL),
     (dict(ms=None), B.EINVAL), (dict(variant=B.CONST), B.EINVAL),          # ms given to the constant variant

@@ -292,3 +292,42 @@ def test_delay_compensated_synchronous_rounds():
         U.assert_state_equal(gpu, cpu)
     (p,) = B.plan_log(ev[: 2 * M], M, 2 * M, wl.eta)
     assert p.n_slots == 1 and p.n_snapshot_reads == 0 and p.n_stores == M      # one shared in-window snapshot
+
+
+@pytest.mark.parametrize("K", [1, 8, 32, 1000])
+@pytest.mark.parametrize("n", [3, 1023, 70_001])
+@pytest.mark.parametrize("adaptive,bf16", [(False, False), (True, False), (False, True), (True, True)])
+def test_momentum_variant(K, n, adaptive, bf16):
+    """Momentum variant (v = beta*v + eta*u ; w = w - v): single messages and fused windows equal
+    the checker bit for bit, velocity included; beta = 0 equals the server without momentum."""
+    wl = small_workload(n, adaptive, bf16, M=6, pushes=90, G=10, seed=K)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    gpu, cpu = U.gpu_server(wl, w0, beta=0.9), U.cpu_server(wl, w0, beta=0.9)
+    gpu.pull(1)
+    gpu.push(1, dpool[2], 0.05)
+    cpu.pull(1)
+    cpu.push(1, pool[2, :n], np.float32(0.05))
+    gpu.apply_log(ev, dpool, K)
+    cpu.replay(ev, pool[:, :n])
+    U.assert_state_equal(gpu, cpu, what=f"momentum K={K} ")
+    zero, plain = U.gpu_server(wl, w0, beta=0.0), U.gpu_server(wl, w0)
+    zero.apply_log(ev, dpool, K)
+    plain.apply_log(ev, dpool, K)
+    import torch
+    torch.cuda.synchronize()
+    assert torch.equal(zero.w, plain.w) and torch.equal(zero.w_bak, plain.w_bak)
+
+
+def test_momentum_checkpoint_carries_the_velocity():
+    wl = small_workload(9_001, True, False, M=4, pushes=60, G=7)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    first = U.gpu_server(wl, w0, beta=0.5)
+    first.apply_log(ev[:51], dpool, 16)
+    ckpt = first.state_dict()
+    resumed = B.Server(None, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, wl.bf16_grad, state=ckpt, beta=0.5)
+    resumed.apply_log(ev[51:], dpool, 16)
+    cpu = U.cpu_server(wl, w0, beta=0.5)
+    cpu.replay(ev, pool[:, : wl.n])
+    U.assert_state_equal(resumed, cpu)

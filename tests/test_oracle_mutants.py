@@ -33,6 +33,10 @@ MUTANTS = [
     ("gradient_buffer_0", "grads + (uint64_t)r.grad_id * grad_stride", "grads", 0),
     ("record_eta_ignored", "r.eta < 0.0f ? default_eta : (T)r.eta", "default_eta", 0),
     ("bf16_widened_wrong", "(uint32_t)h << 16", "(uint32_t)h << 15", 0),
+    ("momentum_decay_dropped", "T bv = beta * vel[i];", "T bv = vel[i];", 0),
+    ("momentum_velocity_not_kept", "vel[i] = nv;", "", 0),
+    ("momentum_step_ignores_velocity", "p = nv;", "", 0),
+    ("momentum_adds_old_velocity_twice", "T nv = bv + p;", "T nv = bv + p + bv;", 0),
     ("one_minus_mu_is_one", "const T omm = (T)1 - mu;", "const T omm = (T)1;", 0),
 ]
 

@@ -317,9 +317,62 @@ def pin_delay_compensated_ssgd(L):
         assert [Fr(float(x)) for x in s.w] == w
 
 
+def pin_momentum(L):
+    """Momentum reading v = beta*v + eta*u ; w = w - v (u = the delay-compensated gradient):
+    beta = 0 is the plain update bit for bit; with lambda = 0 and no delay it is textbook
+    heavy-ball SGD (independent numpy loop, bit for bit); with dyadic inputs the binary64
+    checker equals the recursion over the rationals exactly; the velocity starts at 0 and a
+    pull does not touch it."""
+    f = np.float32
+    for adaptive, lam in ((False, 0.04), (True, 2.0)):
+        ev, w0, grads = _random_case(31, n=130, pushes=40)
+        plain = oracle.Server(w0, 4, adaptive, 0.1, lam, 0.95, 1e-7, library=L)
+        zero = oracle.Server(w0, 4, adaptive, 0.1, lam, 0.95, 1e-7, library=L, beta=0.0)
+        some = oracle.Server(w0, 4, adaptive, 0.1, lam, 0.95, 1e-7, library=L, beta=0.9)
+        for s in (plain, zero, some):
+            s.replay(ev, grads)
+        assert np.array_equal(plain.w, zero.w) and np.array_equal(plain.w_bak, zero.w_bak)
+        assert not np.array_equal(plain.w, some.w)
+    # textbook momentum SGD: lambda = 0, pull right before every push
+    ev, w0, grads = _random_case(32, proto=synth.PROTO_TAU0)
+    s = oracle.Server(w0, 4, False, 0.1, 0.0, library=L, beta=f(0.9))
+    assert np.all(s.v == 0)
+    s.replay(ev, grads)
+    w, v = w0.copy(), np.zeros_like(w0)
+    for r in ev[ev["kind"] == PUSH]:
+        v = f(0.9) * v + f(r["eta"]) * grads[r["grad_id"]]
+        w = w - v
+    assert np.array_equal(s.w, w) and np.array_equal(s.v, v)
+    # exact rational recursion with delays and compensation, dyadic inputs, binary64
+    rng = np.random.default_rng(33)
+    n, M, P = 4, 3, 6
+    w0 = rng.integers(-16, 17, n) / 8.0
+    g = rng.choice([-1.0, -0.5, 0.5, 1.0], size=(P, n))
+    recs = []
+    for e in range(P):
+        recs += [(PUSH, int(rng.integers(M)), e, 0.5), (PULL, int(rng.integers(M)))]
+    ev = synth.make_log(recs)
+    beta, eta, lam = Fr(1, 2), Fr(1, 2), Fr(1)
+    s = oracle.Server(w0, M, False, float(eta), float(lam), dtype=np.float64, library=L, beta=float(beta))
+    s.replay(ev, np.ascontiguousarray(g))
+    w = [Fr(x) for x in w0]
+    wb = [list(w) for _ in range(M)]
+    v = [Fr(0)] * n
+    for r in ev:
+        m = int(r["worker"])
+        if r["kind"] == PULL:
+            wb[m] = list(w)
+            continue
+        gi = [Fr(float(x)) for x in g[int(r["grad_id"])]]
+        u = [gi[i] + lam * gi[i] * gi[i] * (w[i] - wb[m][i]) for i in range(n)]
+        v = [beta * v[i] + eta * u[i] for i in range(n)]
+        w = [w[i] - v[i] for i in range(n)]
+    assert [Fr(float(x)) for x in s.w] == w and [Fr(float(x)) for x in s.v] == v
+
+
 PINS = [pin_hand_constant, pin_closed_form_repeated, pin_hand_adaptive, pin_exact_rational_replay,
         pin_lambda0_is_asgd, pin_tau0_is_sgd, pin_meansquare_unrolled, pin_adaptive_lambda_definition,
-        pin_protocol, pin_bruteforce_f32, pin_f32_tracks_f64, pin_delay_compensated_ssgd]
+        pin_protocol, pin_bruteforce_f32, pin_f32_tracks_f64, pin_delay_compensated_ssgd, pin_momentum]
 
 
 @pytest.mark.parametrize("pin", PINS, ids=lambda p: p.__name__)
