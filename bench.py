@@ -50,7 +50,7 @@ FALLBACK_HBM_GBS = 6650.0
 # of the benchmark by its algorithmic bytes.  Tied to the kernel sources by hash: a changed kernel
 # voids the figure (reported as null).  Summary: profiles/k_replay_adaptive_f32_c3_window32.md
 NCU_TRAFFIC: dict[str, dict] = {
-    "k_replay<adaptive,f32>": {"src": "424ff788e326e444", "dram_bytes_per_algorithmic_byte": 0.9895},
+    "k_replay<adaptive,f32>": {"src": "e0f806aecbe4ea5e", "dram_bytes_per_algorithmic_byte": 0.9895},
 }
 
 

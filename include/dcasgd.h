@@ -197,8 +197,7 @@ typedef struct {
 int dcasgd_compile_window(const dcasgd_event *ev, uint64_t count, uint32_t num_workers, uint32_t window_k,
                           float default_eta, uint32_t max_slots, dcasgd_window_program *out);
 
-/* The slot limit dcasgd_apply_log passes to the compiler for this server (it keeps the shared
- * memory of a window small enough for two or more CTAs per SM): with it,
+/* The slot limit dcasgd_apply_log passes to the compiler for this server: with it,
  * dcasgd_compile_window cuts a log exactly as dcasgd_apply_log does. */
 int dcasgd_get_window_slot_cap(const dcasgd_server *s, uint32_t *max_slots);
 

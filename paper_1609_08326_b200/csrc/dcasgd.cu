@@ -18,8 +18,9 @@ struct dcasgd_server {
     Hyper h;
     cudaStream_t stream;
     int device;
-    int replay_vecs;     // 16-byte vectors per thread in the fused replay kernel (1 or 2)
-    uint32_t slot_cap;   // in-window snapshot slots a window may use (keeps >= 2 CTAs per SM resident)
+    int replay_vecs;     // 16-byte vectors per thread in the fused replay kernel (1 or 2) for windows with few slots
+    uint32_t two_vec_slots;  // a window that needs more slots than this runs one vector per thread
+    uint32_t slot_cap;   // in-window snapshot slots a window may use
     uint64_t t;          // pushes applied (Algorithm 2's t)
     uint64_t launches;   // kernels launched through this handle
 };
@@ -153,7 +154,8 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.grad_pool = static_cast<const char*>(grad_pool);
     a.n = c.n;
     a.h = s->h;
-    const int V = s->replay_vecs;
+    // many live snapshots: one vector per thread keeps two CTAs per SM resident (a slot costs half)
+    const int V = wp.n_slots > s->two_vec_slots ? 1 : s->replay_vecs;
     const unsigned grid = blocks_for(c.n, V);
     const size_t smem = replay_smem_bytes(wp.n_slots, V);
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
@@ -304,9 +306,11 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->replay_vecs = blocks_for(c.n, 2) >= 2u * (unsigned)sms ? 2 : 1;
     if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) { const int k = std::atoi(v); if (k == 1 || k == 2) s->replay_vecs = k; }
     // A slot costs 4 KB (8 KB with two vectors per thread) of shared memory per CTA on top of the
-    // staging ring.  Long windows over many workers would take all 16 slots and leave one CTA
-    // per SM; capping the slots cuts such a window a little earlier and keeps two or more resident.
-    s->slot_cap = 8;
+    // staging ring.  Windows that keep up to 8 snapshots run two vectors per thread (2-3 CTAs per
+    // SM); longer windows over many workers need up to 16 and run one vector per thread (2 CTAs
+    // per SM), which measured faster than cutting them at 8 slots.
+    s->two_vec_slots = 8;
+    s->slot_cap = DCASGD_MAX_WINDOW_SLOTS;
     if (const char* v = std::getenv("DCASGD_WINDOW_SLOTS")) { const int k = std::atoi(v); if (k >= 1 && k <= DCASGD_MAX_WINDOW_SLOTS) s->slot_cap = (uint32_t)k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
