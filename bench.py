@@ -12,7 +12,7 @@ element-updates per second = parameters x pushes / time.  Inputs are synthetic a
 
 Printed: ONE JSON line (rank 0).  Besides the headline it carries
   roofline      the dominant kernel (fused window replay) against measured HBM copy bandwidth
-  variants      the same log replayed with windows of 8 records and unfused (one kernel per message)
+  variants      the same log replayed with windows of 8 and of 256 records and unfused (one kernel per message)
   kernels       single push / single pull kernels timed on their own (50 launches each)
   e2e           the same metric with host buffers: pinned host -> device copies of the model and
                 the gradient pool, replay, and the model copied back, all inside the timed region
@@ -370,7 +370,7 @@ def run_b200(args) -> None:
 
     if not args.headline_only:
         variants = {}
-        for name, wk in (("fused_k8", 8), ("unfused_k1", 1)):
+        for name, wk in (("fused_k8", 8), ("fused_k256", 256), ("unfused_k1", 1)):
             if wk == args.window_k:
                 continue
             t_ms, r_ms, ps = replay_steps(wk, K, W)
