@@ -279,6 +279,9 @@ class Server:
                 self.v.copy_(state["v"])
         self.bf16_grad = bool(bf16_grad)
         self.stream = stream
+        if stream is not None:
+            # the copies above ran on torch's current stream; the server's kernels run on `stream`
+            stream.wait_stream(torch.cuda.current_stream(self.device))
         s = stream.cuda_stream if stream is not None else torch.cuda.current_stream(self.device).cuda_stream
         with torch.cuda.device(self.device):
             self.h = dcasgd_create(self.n, self.M, ADAPTIVE if adaptive else CONST, BF16 if bf16_grad else F32,

@@ -74,6 +74,57 @@ int check_foreign(const dcasgd_config& c, const void* p, uint64_t bytes, const c
     return DCASGD_OK;
 }
 
+// cuMemGetAddressRange of the driver, looked up through the runtime (the library does not link
+// against the driver); NULL when the lookup fails, and the extent check is then skipped.
+typedef int (*mem_range_fn)(unsigned long long* base, size_t* size, unsigned long long ptr);
+mem_range_fn mem_range() {
+    static const mem_range_fn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuMemGetAddressRange", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            f = nullptr;
+        }
+        return reinterpret_cast<mem_range_fn>(f);
+    }();
+    return fn;
+}
+
+// One address must be device (or managed) memory of device `dev`.
+int check_device_address(const char* fn, const char* name, const void* p, int dev) {
+    cudaPointerAttributes at;
+    const cudaError_t e = cudaPointerGetAttributes(&at, p);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return fail(DCASGD_EINVAL, "%s: %s is not a usable device pointer (%s)", fn, name, cudaGetErrorName(e)); }
+    if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged)
+        return fail(DCASGD_EINVAL, "%s: %s is not device memory", fn, name);
+    if (at.type == cudaMemoryTypeDevice && at.device != dev)
+        return fail(DCASGD_EINVAL, "%s: %s lives on device %d, current device is %d", fn, name, at.device, dev);
+    return DCASGD_OK;
+}
+
+// A caller buffer [p, p+bytes) must be device memory of device `dev` from its first to its last
+// byte: a host pointer, another device's memory or a buffer shorter than stated is refused here,
+// on the host, instead of faulting in a kernel.  The extent is checked against the allocation
+// that holds p; a buffer that spans several mappings (a virtual-memory pool) is accepted when
+// its last byte is device memory of the same device too.
+int check_device_buffer(const char* fn, const char* name, const void* p, uint64_t bytes, int dev) {
+    if (bytes == 0) return DCASGD_OK;
+    int rc = check_device_address(fn, name, p, dev);
+    if (rc) return rc;
+    const char* last = static_cast<const char*>(p) + (bytes - 1);
+    if (mem_range_fn range = mem_range()) {
+        unsigned long long base = 0;
+        size_t size = 0;
+        if (range(&base, &size, (unsigned long long)reinterpret_cast<uintptr_t>(p)) == 0 &&
+            reinterpret_cast<uintptr_t>(last) < base + size)
+            return DCASGD_OK;
+    }
+    if (check_device_address(fn, name, last, dev))
+        return fail(DCASGD_EINVAL, "%s: %s is shorter than the %llu bytes this call needs", fn, name, (unsigned long long)bytes);
+    return DCASGD_OK;
+}
+
 inline unsigned blocks_for(uint64_t n, int vecs_per_thread) {
     const uint64_t nvec = (n + 3) / 4;
     const uint64_t per_block = (uint64_t)kThreads * vecs_per_thread;
@@ -97,8 +148,7 @@ int launch_pull(dcasgd_server* s, uint32_t m, float* out_w) {
 
 int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
     const dcasgd_config& c = s->cfg;
-    s->t += 1;
-    if (c.n == 0) return DCASGD_OK;
+    if (c.n == 0) { s->t += 1; return DCASGD_OK; }
     PushArgs a;
     a.w = c.w;
     a.wb_m = c.w_bak + (uint64_t)m * c.w_bak_stride;
@@ -120,30 +170,38 @@ int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
     else if (bf)        DCASGD_LAUNCH_PUSH(false, true);
     else                DCASGD_LAUNCH_PUSH(false, false);
 #undef DCASGD_LAUNCH_PUSH
-    return after_launch(s, "push kernel");
+    const int rc = after_launch(s, "push kernel");
+    if (rc == DCASGD_OK) s->t += 1;              // t counts the pushes that were actually enqueued
+    return rc;
 }
 
 int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void* grad_pool,
                   uint64_t grad_stride_bytes) {
     const dcasgd_config& c = s->cfg;
-    s->t += wp.n_pushes;
-    if (c.n == 0) return DCASGD_OK;
+    if (c.n == 0) { s->t += wp.n_pushes; return DCASGD_OK; }
     if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
-    static thread_local DevProgram p;            // 4.6 KB: kept off the stack
+    // many live snapshots: one vector per thread keeps two CTAs per SM resident (a slot costs half)
+    const int V = wp.n_slots > s->two_vec_slots ? 1 : s->replay_vecs;
+    const int S = replay_stages(V);
+    static thread_local DevProgram p;            // 5.6 KB: kept off the stack
     std::memset(&p, 0, sizeof p);
     p.n_pushes = wp.n_pushes;
-    p.n_slots = wp.n_slots;
-    p.save_slot0 = (int8_t)wp.save_slot[0];
-    p.store_end0 = (uint8_t)wp.store_begin[1];
+    p.save_off0 = wp.save_slot[0] >= 0 ? replay_slot_off(V, (uint32_t)wp.save_slot[0]) : kNoSave;
+    p.store_end0 = wp.store_begin[1];
     for (uint32_t j = 0; j < wp.n_pushes; ++j) {
         FetchStep& f = p.fetch[j];
         ApplyStep& ap = p.apply[j];
         f.g_off = (uint64_t)wp.grad_id[j] * grad_stride_bytes;
         ap.eta = wp.eta[j];
-        if (wp.src[j] >= 0) { ap.src_slot = -1; f.s_off = (uint64_t)wp.src[j] * c.w_bak_stride * 4; }
-        else                { ap.src_slot = (int8_t)(-(wp.src[j] + 1)); f.s_off = kNoMemorySnapshot; }
-        ap.save_slot = (int8_t)wp.save_slot[j + 1];
-        ap.store_end = (uint8_t)wp.store_begin[j + 2];
+        if (wp.src[j] >= 0) {                    // staged from memory into this push's stage of the snapshot ring
+            f.s_off = (uint64_t)wp.src[j] * c.w_bak_stride * 4;
+            ap.snap_off = replay_snap_ring_off(V, j % (uint32_t)S);
+        } else {                                 // an in-window slot
+            f.s_off = kNoMemorySnapshot;
+            ap.snap_off = replay_slot_off(V, (uint32_t)(-(wp.src[j] + 1)));
+        }
+        ap.save_off = wp.save_slot[j + 1] >= 0 ? replay_slot_off(V, (uint32_t)wp.save_slot[j + 1]) : kNoSave;
+        ap.store_end = wp.store_begin[j + 2];
     }
     for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_off[k] = (uint64_t)wp.store_worker[k] * c.w_bak_stride * 4;
     ReplayArgs a;
@@ -154,8 +212,6 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.grad_pool = static_cast<const char*>(grad_pool);
     a.n = c.n;
     a.h = s->h;
-    // many live snapshots: one vector per thread keeps two CTAs per SM resident (a slot costs half)
-    const int V = wp.n_slots > s->two_vec_slots ? 1 : s->replay_vecs;
     const unsigned grid = blocks_for(c.n, V);
     const size_t smem = replay_smem_bytes(wp.n_slots, V);
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
@@ -174,7 +230,9 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     else if (bf)        DCASGD_LAUNCH_REPLAY(false, true);
     else                DCASGD_LAUNCH_REPLAY(false, false);
 #undef DCASGD_LAUNCH_REPLAY
-    return after_launch(s, "window replay kernel");
+    const int rc = after_launch(s, "window replay kernel");
+    if (rc == DCASGD_OK) s->t += wp.n_pushes;
+    return rc;
 }
 
 template <bool AD, bool BF, bool MOM>
@@ -265,17 +323,11 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return cuda_fail("dcasgd_create: cudaGetDevice", e);
     if (c.n) {
-        const void* ptrs[4] = {c.w, c.w_bak, c.ms, c.v};
-        const char* names[4] = {"w", "w_bak", "ms", "v"};
-        for (int i = 0; i < 4; ++i) {
-            if (!ptrs[i]) continue;
-            cudaPointerAttributes at;
-            e = cudaPointerGetAttributes(&at, ptrs[i]);
-            if (e != cudaSuccess) return cuda_fail("dcasgd_create: cudaPointerGetAttributes", e);
-            if (at.type != cudaMemoryTypeDevice && at.type != cudaMemoryTypeManaged)
-                return fail(DCASGD_EINVAL, "dcasgd_create: %s is not device memory", names[i]);
-            if (at.type == cudaMemoryTypeDevice && at.device != dev)
-                return fail(DCASGD_EINVAL, "dcasgd_create: %s lives on device %d, current device is %d", names[i], at.device, dev);
+        Range st[4];
+        const int k = state_ranges(c, st);
+        for (int i = 0; i < k; ++i) {
+            const int rc = check_device_buffer("dcasgd_create", st[i].name, st[i].lo, (uint64_t)(st[i].hi - st[i].lo), dev);
+            if (rc) return rc;
         }
     }
     if ((e = allow_slots<false, false>()) != cudaSuccess || (e = allow_slots<false, true>()) != cudaSuccess ||
@@ -329,6 +381,7 @@ int dcasgd_pull(dcasgd_server* s, uint32_t m, float* out_w) {
     if (out_w && s->cfg.n) {
         if (!aligned16(out_w)) return fail(DCASGD_EALIGN, "dcasgd_pull: out_w must be 16-byte aligned");
         if ((rc = check_foreign(s->cfg, out_w, s->cfg.n * 4, "out_w"))) return rc;
+        if ((rc = check_device_buffer("dcasgd_pull", "out_w", out_w, s->cfg.n * 4, s->device))) return rc;
     }
     return launch_pull(s, m, out_w);
 }
@@ -342,6 +395,7 @@ int dcasgd_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
         if (!g) return fail(DCASGD_EINVAL, "dcasgd_push: g is NULL");
         if (!aligned16(g)) return fail(DCASGD_EALIGN, "dcasgd_push: g must be 16-byte aligned");
         if ((rc = check_foreign(s->cfg, g, s->cfg.n * grad_elem_bytes(s->cfg), "g"))) return rc;
+        if ((rc = check_device_buffer("dcasgd_push", "g", g, s->cfg.n * grad_elem_bytes(s->cfg), s->device))) return rc;
     }
     return launch_push(s, m, g, eta);
 }
@@ -370,7 +424,9 @@ int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, c
         if (!grad_pool) return fail(DCASGD_EINVAL, "dcasgd_apply_log: grad_pool is NULL");
         if (!aligned16(grad_pool) || grad_stride_bytes % 16) return fail(DCASGD_EALIGN, "dcasgd_apply_log: grad_pool and grad_stride_bytes must be multiples of 16 bytes");
         if (num_grads > 1 && grad_stride_bytes < gbytes) return fail(DCASGD_EINVAL, "dcasgd_apply_log: grad_stride_bytes smaller than one gradient");
-        if ((rc = check_foreign(c, grad_pool, (uint64_t)(num_grads - 1) * grad_stride_bytes + gbytes, "grad_pool"))) return rc;
+        const uint64_t pool_bytes = (uint64_t)(num_grads - 1) * grad_stride_bytes + gbytes;
+        if ((rc = check_foreign(c, grad_pool, pool_bytes, "grad_pool"))) return rc;
+        if ((rc = check_device_buffer("dcasgd_apply_log", "grad_pool", grad_pool, pool_bytes, s->device))) return rc;
     }
 
     if (window_k == 1) {
@@ -420,12 +476,20 @@ int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, voi
     if (!(al >= 0x1p-60f && al < 0x1p60f)) return fail(DCASGD_EINVAL, "dcasgd_check_adaptive_lambda: |lambda0| must be in [2^-60, 2^60)");
     if (!(s_first >= 0x1p-100f && s_last < 0x1p100f && s_first <= s_last))
         return fail(DCASGD_EINVAL, "dcasgd_check_adaptive_lambda: need 2^-100 <= s_first <= s_last < 2^100");
+    if (reinterpret_cast<uintptr_t>(mismatches_dev) & 7u)
+        return fail(DCASGD_EALIGN, "dcasgd_check_adaptive_lambda: mismatches_dev must be 8-byte aligned");
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("dcasgd_check_adaptive_lambda: cudaGetDevice", e);
+    if (const int rc = check_device_buffer("dcasgd_check_adaptive_lambda", "mismatches_dev", mismatches_dev, 8, dev)) return rc;
+    int sms = 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
     uint32_t b0, b1;
     std::memcpy(&b0, &s_first, 4);
     std::memcpy(&b1, &s_last, 4);
-    k_check_lambda<<<148 * 8, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+    k_check_lambda<<<(unsigned)sms * 8, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         lambda0, b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
-    const cudaError_t e = cudaGetLastError();
+    e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("lambda self-check kernel", e);
     return DCASGD_OK;
 }

@@ -126,6 +126,10 @@ int WindowCompiler::compile(const dcasgd_event* ev, uint64_t count, uint32_t win
                             uint32_t max_slots, dcasgd_window_program* out) {
     if (max_slots == 0 || max_slots > DCASGD_MAX_WINDOW_SLOTS) max_slots = DCASGD_MAX_WINDOW_SLOTS;
     uint64_t K = count < window_k ? count : window_k;
+    // A window holds a few hundred pushes and stores at most, and every attempt below walks all K
+    // records: bound K so that compiling a long log with a huge window_k stays linear in the log.
+    // (A shorter window is always legal and the results are the same bit for bit.)
+    if (K > kMaxWindowScan) K = kMaxWindowScan;
     for (uint64_t r = 0; r < K; ++r) {
         if (ev[r].kind > DCASGD_PUSH) { set_error("log record %llu: unknown kind %u", (unsigned long long)r, ev[r].kind); return DCASGD_ELOG; }
         if (ev[r].worker >= M) { set_error("log record %llu: worker %u >= %u", (unsigned long long)r, ev[r].worker, M); return DCASGD_ELOG; }

@@ -12,6 +12,9 @@ namespace dcasgd {
 void set_error(const char* fmt, ...);
 const char* get_error();
 
+// Records one window may span at most, whatever window_k says (see WindowCompiler::compile).
+constexpr uint64_t kMaxWindowScan = 2048;
+
 // Reusable scratch for compiling many windows of one log (per-worker arrays are allocated once).
 struct WindowCompiler {
     explicit WindowCompiler(uint32_t num_workers);

@@ -149,6 +149,34 @@ def test_empty_model_and_side_stream():
     U.assert_state_equal(gpu, cpu)
 
 
+def test_side_stream_with_device_w0_and_resumed_state():
+    """The binding fills w (and, on resume, w_bak / ms) on torch's current stream while the
+    server's kernels run on its own stream: the first kernel must wait for those copies."""
+    import torch
+    wl = small_workload(300_007, True, False, M=5, pushes=60, G=9)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    cpu = U.cpu_server(wl, w0)
+    cpu.replay(ev, pool[:, : wl.n])
+    st = torch.cuda.Stream()
+    w0_dev = torch.from_numpy(w0).cuda()
+    torch.cuda.synchronize()
+    busy = torch.empty(64 << 20, device="cuda")
+    for _ in range(20):
+        busy.normal_()                                   # keeps the current stream busy ahead of the copies
+    gpu = B.Server(w0_dev * 1.0, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, stream=st)
+    a = 41
+    gpu.apply_log(ev[:a], dpool, 16)
+    ckpt = gpu.state_dict()
+    for _ in range(20):
+        busy.normal_()
+    resumed = B.Server(None, wl.M, wl.adaptive, wl.eta, wl.lam, wl.mu, wl.eps, stream=st,
+                       state={k: (v.cuda() if hasattr(v, "cuda") else v) for k, v in ckpt.items()})
+    resumed.apply_log(ev[a:], dpool, 16)
+    st.synchronize()
+    U.assert_state_equal(resumed, cpu)
+
+
 def test_errors_leave_the_state_untouched():
     import torch
     wl = small_workload(1000, True, False, M=4)
@@ -183,6 +211,40 @@ def test_errors_leave_the_state_untouched():
     assert gpu.launches == launches and gpu.step == 0
     for a, b in zip(before, (gpu.w, gpu.w_bak_buf, gpu.ms)):
         assert torch.equal(a, b)
+    # per-call buffers that are not device memory of the server's GPU, or shorter than the call
+    # needs, are refused on the host: nothing is launched, so no bad address ever reaches a kernel
+    host_g = torch.zeros(1024).pin_memory()
+    plain = np.zeros(1024, dtype=np.float32)
+    expect(B.EINVAL, lambda: gpu.push(0, host_g))
+    expect(B.EINVAL, lambda: gpu.push(0, plain))
+    expect(B.EINVAL, lambda: gpu.pull(0, host_g))
+    expect(B.EINVAL, lambda: gpu.apply_log(synth.make_log(good[:2]), host_g, 8, grad_stride_bytes=4096, num_grads=1))
+    try:                                                 # an allocation of exactly 4000 bytes, outside torch's pools
+        from cuda.bindings import runtime as cudart
+    except ImportError:
+        cudart = None
+    if cudart is not None:
+        err, raw = cudart.cudaMalloc(4000)
+        assert int(err) == 0
+        try:
+            gpu_ok = U.gpu_server(wl, w0)
+            torch.cuda.synchronize()
+            n_before = gpu_ok.launches
+            gpu_ok.push(0, int(raw))                     # 1000 floats fit exactly
+            assert gpu_ok.launches == n_before + 1
+            expect(B.EINVAL, lambda: gpu_ok.push(0, int(raw) + 2048))        # 1952 bytes left: too short
+            expect(B.EINVAL, lambda: gpu_ok.pull(0, int(raw) + 2048))
+            expect(B.EINVAL, lambda: gpu_ok.apply_log(synth.make_log(good), int(raw), 8, grad_stride_bytes=4000, num_grads=2))
+            gpu_ok.apply_log(synth.make_log(good[:2]), int(raw), 8, grad_stride_bytes=4000, num_grads=1)   # exactly one buffer fits
+            assert gpu_ok.launches == n_before + 2
+            torch.cuda.synchronize()
+        finally:
+            cudart.cudaFree(raw)
+    counter = torch.zeros(2, dtype=torch.int64, device="cuda")
+    expect(B.EALIGN, lambda: B.dcasgd_check_adaptive_lambda(2.0, 1.0, 2.0, counter.data_ptr() + 4))
+    expect(B.EINVAL, lambda: B.dcasgd_check_adaptive_lambda(2.0, 1.0, 2.0, np.zeros(1, dtype=np.int64)))
+    torch.cuda.synchronize()
+    assert gpu.launches == launches and gpu.step == 0 and int(counter.sum().item()) == 0
     # host memory handed in as state is refused
     host = torch.zeros(1000)
     with pytest.raises(B.DcasgdError):

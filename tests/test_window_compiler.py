@@ -163,3 +163,17 @@ def test_slot_cap_cuts_windows_but_not_results(cap):
         assert [p.n_records for p in progs] == [p.n_records for p in full]
     with pytest.raises(B.DcasgdError):
         B.dcasgd_compile_window(ev, 16, 8, 0.1, max_slots=17)
+
+
+def test_huge_window_k_stays_linear_in_the_log():
+    """window_k far beyond what a window can hold: the compiler bounds the records it scans per
+    window, so planning a long log takes time proportional to the log (and cuts it correctly)."""
+    import time
+    ev = synth.event_log(16, 60_000, synth.ORDER_UNIFORM, synth.PROTO_ASYNC, 5, 0.1, seed=11)
+    t0 = time.perf_counter()
+    progs = B.plan_log(ev, 16, 2 ** 32 - 1, 0.1)
+    dt = time.perf_counter() - t0
+    assert sum(p.n_records for p in progs) == len(ev)
+    assert all(p.n_records <= 2048 for p in progs)
+    assert dt < 20.0, f"planning {len(ev)} records took {dt:.1f} s"
+    check(ev[:3000], 16, 2 ** 32 - 1)
