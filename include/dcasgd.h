@@ -158,6 +158,20 @@ uint32_t dcasgd_version(void);
  * The expected count is 0 for every admissible argument. */
 int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, void *stream, uint64_t *mismatches_dev);
 
+/* Checked build, no counterpart in the paper.  A library compiled with -DDCASGD_DEBUG_CHECKS
+ * makes every kernel compare each global-memory address it is about to use with the buffers of
+ * the call (the server's w / w_bak / ms / v and the caller's g, out_w or gradient pool, with the
+ * extents the host validated).  An access outside all of them, a store into a read-only buffer
+ * or a misaligned access is skipped - nothing traps, nothing faults - and a bit is ORed into
+ * *status_dev (device, 4 bytes, 4-byte aligned, zeroed by the caller): 1 = bad read,
+ * 2 = bad write, 4 = misaligned.  With a server handle the word serves that server from its
+ * next launch on; with s = NULL it becomes the default that servers created afterwards (and the
+ * lambda self-check) inherit, so that "Initialize" is covered too.  status_dev = NULL stops the
+ * recording (violating accesses are still skipped).  The access table sits in constant memory
+ * and is replaced in stream order before each launch: use one stream at a time in this build.
+ * In the normal build no check exists in the kernels and this call returns DCASGD_EINVAL. */
+int dcasgd_debug_checks(dcasgd_server *s, uint32_t *status_dev);
+
 /* ---- window compiler (host only; no CUDA call) -------------------------------------------
  * What dcasgd_apply_log does to a window before launching, exposed so that it can be
  * inspected and tested without a GPU.  A window of the log becomes a list of STEPS.  Step 0 has

@@ -19,6 +19,7 @@ import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "csrc", "libdcasgd.so")
+DEBUG_LIB_PATH = os.path.join(HERE, "csrc", "libdcasgd_checked.so")    # the -DDCASGD_DEBUG_CHECKS build
 
 OK, EINVAL, EWORKER, EALIGN, ELOG, ECUDA, ENOMEM = range(7)
 CONST, ADAPTIVE = 0, 1
@@ -31,7 +32,7 @@ MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
 SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
            "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_last_error",
            "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window", "dcasgd_check_adaptive_lambda",
-           "dcasgd_get_window_slot_cap"]
+           "dcasgd_get_window_slot_cap", "dcasgd_debug_checks"]
 
 
 class Config(C.Structure):
@@ -65,10 +66,13 @@ def lib() -> C.CDLL:
     """Loads csrc/libdcasgd.so (building it in-tree first if it is absent and nvcc exists)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
+        # DCASGD_CHECKED_BUILD=1 selects the library whose kernels bounds-check every access
+        checked = os.environ.get("DCASGD_CHECKED_BUILD", "0") == "1"
+        path = DEBUG_LIB_PATH if checked else LIB_PATH
+        if not os.path.exists(path):
             from . import build
-            build.build_lib()
-        L = C.CDLL(LIB_PATH)
+            build.build_lib(debug_checks=checked)
+        L = C.CDLL(path)
         u64, u32, vp = C.c_uint64, C.c_uint32, C.c_void_p
         L.dcasgd_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
         L.dcasgd_pull.argtypes = [vp, u32, vp]
@@ -83,6 +87,8 @@ def lib() -> C.CDLL:
         L.dcasgd_get_window_slot_cap.restype = C.c_int
         L.dcasgd_check_adaptive_lambda.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp]
         L.dcasgd_check_adaptive_lambda.restype = C.c_int
+        L.dcasgd_debug_checks.argtypes = [vp, vp]
+        L.dcasgd_debug_checks.restype = C.c_int
         for name in ("dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
                      "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_compile_window"):
             getattr(L, name).restype = C.c_int
@@ -188,6 +194,11 @@ def dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, mismatches_dev, strea
     """Adds to the device counter the number of s in [s_first, s_last] on which the two routes
     of lambda_0 / sqrt(s) differ (expected: 0)."""
     _check(lib().dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, stream, _ptr(mismatches_dev)))
+
+
+def dcasgd_debug_checks(h, status_dev) -> None:
+    """Checked build only: the device word that collects access violations (see dcasgd.h)."""
+    _check(lib().dcasgd_debug_checks(h, _ptr(status_dev)))
 
 
 def plan_log(ev, num_workers, window_k, default_eta=0.0, max_slots=0) -> list[WindowProgram]:

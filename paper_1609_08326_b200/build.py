@@ -3,10 +3,12 @@
     python -m paper_1609_08326_b200.build          # everything
     python -m paper_1609_08326_b200.build synth    # only the input generator
     python -m paper_1609_08326_b200.build lib      # only the CUDA server library
+    python -m paper_1609_08326_b200.build checked  # only its bounds-checked twin
 
 Outputs (git-ignored shared objects next to their sources):
     synth/libdcasgd_synth.so   g++,  seeded input generator (host only)
     csrc/libdcasgd.so          nvcc, sm_100a, the C-ABI server library declared in include/dcasgd.h
+    csrc/libdcasgd_checked.so  the same sources with -DDCASGD_DEBUG_CHECKS (bounds-checked kernels; tests only)
 """
 from __future__ import annotations
 
@@ -26,6 +28,7 @@ LIB_HDRS = [os.path.join(PKG, "csrc", "window_compiler.h"),
             os.path.join(PKG, "csrc", "kernels.cuh"),
             os.path.join(ROOT, "include", "dcasgd.h")]
 LIB_SO = os.path.join(PKG, "csrc", "libdcasgd.so")
+LIB_CHECKED_SO = os.path.join(PKG, "csrc", "libdcasgd_checked.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -68,20 +71,26 @@ def nvcc_path() -> str:
     return cand
 
 
-def build_lib(force: bool = False, verbose_ptxas: bool = False) -> str:
-    if force or _stale(LIB_SO, LIB_SRCS + LIB_HDRS + [os.path.abspath(__file__)]):
+def build_lib(force: bool = False, verbose_ptxas: bool = False, debug_checks: bool = False) -> str:
+    """debug_checks: the checked build (libdcasgd_checked.so) whose kernels compare every global
+    address with the buffers of the call, skip what lies outside and report it in a status word."""
+    so = LIB_CHECKED_SO if debug_checks else LIB_SO
+    if force or _stale(so, LIB_SRCS + LIB_HDRS + [os.path.abspath(__file__)]):
         cmd = [nvcc_path(), *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"),
                "-I", os.path.join(PKG, "csrc")]
+        if debug_checks:
+            cmd += ["-DDCASGD_DEBUG_CHECKS"]
         if verbose_ptxas:
             cmd += ["-Xptxas", "-v"]
-        cmd += ["-o", LIB_SO, *LIB_SRCS]
+        cmd += ["-o", so, *LIB_SRCS]
         _run(cmd)
-    return LIB_SO
+    return so
 
 
 def build_all(force: bool = False) -> None:
     build_synth(force)
     build_lib(force)
+    build_lib(force, debug_checks=True)
 
 
 if __name__ == "__main__":
@@ -91,6 +100,8 @@ if __name__ == "__main__":
         print(build_synth(force))
     elif what == "lib":
         print(build_lib(force, verbose_ptxas="-v" in sys.argv))
+    elif what == "checked":
+        print(build_lib(force, verbose_ptxas="-v" in sys.argv, debug_checks=True))
     else:
         build_all(force)
         print(SYNTH_SO)

@@ -23,6 +23,7 @@ struct dcasgd_server {
     uint32_t slot_cap;   // in-window snapshot slots a window may use
     uint64_t t;          // pushes applied (Algorithm 2's t)
     uint64_t launches;   // kernels launched through this handle
+    uint32_t* debug_status;  // checked build: device word that collects access violations, or NULL
 };
 
 namespace {
@@ -131,6 +132,47 @@ inline unsigned blocks_for(uint64_t n, int vecs_per_thread) {
     return (unsigned)((nvec + per_block - 1) / per_block);
 }
 
+#ifdef DCASGD_DEBUG_CHECKS
+uint32_t* g_default_debug_status = nullptr;      // inherited by servers created afterwards
+
+// Checked build: before a launch, tell the kernels which address ranges they may touch - the
+// server's state arrays (writable) and the caller buffer of this call.  The table lives in
+// constant memory and is replaced in stream order, so launches of one stream see their own.
+int debug_arm(cudaStream_t stream, const dcasgd_config* c, uint32_t* status, const void* extra, uint64_t extra_bytes,
+              bool extra_writable) {
+    DebugTable t;
+    std::memset(&t, 0, sizeof t);
+    auto add = [&t](const void* p, uint64_t bytes, bool writable) {
+        if (!p || !bytes) return;
+        t.lo[t.n_ranges] = static_cast<const char*>(p);
+        t.hi[t.n_ranges] = static_cast<const char*>(p) + bytes;
+        if (writable) t.writable |= 1u << t.n_ranges;
+        t.n_ranges += 1;
+    };
+    if (c) {
+        Range st[4];
+        const int k = state_ranges(*c, st);
+        for (int i = 0; i < k; ++i) add(st[i].lo, (uint64_t)(st[i].hi - st[i].lo), true);
+    }
+    add(extra, extra_bytes, extra_writable);
+    // Self-test of the checker: DCASGD_CHECKED_SHRINK=<bytes> makes the TABLE (not the buffers)
+    // that much shorter at the end of every range, so the kernels' legitimate last accesses are
+    // reported and skipped.  No invalid address is ever touched.
+    if (const char* v = std::getenv("DCASGD_CHECKED_SHRINK")) {
+        const long k = std::atol(v);
+        for (uint32_t i = 0; i < t.n_ranges; ++i)
+            if (k > 0 && t.hi[i] - t.lo[i] > k) t.hi[i] -= k;
+    }
+    t.status = status;
+    const cudaError_t e = cudaMemcpyToSymbolAsync(c_dbg, &t, sizeof t, 0, cudaMemcpyHostToDevice, stream);
+    return e == cudaSuccess ? DCASGD_OK : cuda_fail("checked build: arming the access table", e);
+}
+#define DCASGD_DEBUG_ARM(s, extra, bytes, writable)                                                         \
+    do { const int rc_ = debug_arm((s)->stream, &(s)->cfg, (s)->debug_status, extra, bytes, writable); if (rc_) return rc_; } while (0)
+#else
+#define DCASGD_DEBUG_ARM(s, extra, bytes, writable) do { } while (0)
+#endif
+
 int after_launch(dcasgd_server* s, const char* what) {
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(what, e);
@@ -141,6 +183,7 @@ int after_launch(dcasgd_server* s, const char* what) {
 int launch_pull(dcasgd_server* s, uint32_t m, float* out_w) {
     const dcasgd_config& c = s->cfg;
     if (c.n == 0) return DCASGD_OK;
+    DCASGD_DEBUG_ARM(s, out_w, c.n * 4, true);
     k_pull<<<blocks_for(c.n, kPullUnroll), kThreads, 0, s->stream>>>(
         c.w, c.w_bak + (uint64_t)m * c.w_bak_stride, out_w, c.n);
     return after_launch(s, "pull kernel");
@@ -160,6 +203,7 @@ int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
     a.h = s->h;
     const unsigned grid = blocks_for(c.n, kPushUnroll);
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
+    DCASGD_DEBUG_ARM(s, g, c.n * grad_elem_bytes(c), false);
 #define DCASGD_LAUNCH_PUSH(AD, BF)                                                           \
     do {                                                                                     \
         if (mom) k_push<AD, BF, true><<<grid, kThreads, 0, s->stream>>>(a);                  \
@@ -176,7 +220,7 @@ int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
 }
 
 int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void* grad_pool,
-                  uint64_t grad_stride_bytes) {
+                  uint64_t grad_stride_bytes, uint64_t pool_bytes) {
     const dcasgd_config& c = s->cfg;
     if (c.n == 0) { s->t += wp.n_pushes; return DCASGD_OK; }
     if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
@@ -214,6 +258,8 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     a.h = s->h;
     const unsigned grid = blocks_for(c.n, V);
     const size_t smem = replay_smem_bytes(wp.n_slots, V);
+    DCASGD_DEBUG_ARM(s, grad_pool, pool_bytes, false);
+    (void)pool_bytes;
     const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
 #define DCASGD_LAUNCH_REPLAY(AD, BF)                                                         \
     do {                                                                                     \
@@ -342,13 +388,23 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     s->h.omm = 1.0f - s->h.mu;
     s->h.eps = adaptive ? c.eps : 0.0f;
     s->h.beta = c.v ? c.beta : 0.0f;
+    // Route of the adaptive lambda (see kernels.cuh).  The branch-free route is exact for
+    // |lambda_0| in [2^-60, 2^60) and s in [2^-100, 2^100).  The lower bound on s needs no test when
+    // eps >= 2^-100 and MeanSquare starts at 0 here (it is a sum of non-negative terms from then
+    // on); a resumed state comes from the caller, so its MeanSquare is not taken on trust.
     const float al = std::fabs(c.lambda);
-    s->h.fast = (al >= 0x1p-60f && al < 0x1p60f) ? 1u : 0u;
-    if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) s->h.fast = 0u; }
+    s->h.fast = kLambdaLibrary;
+    if (al >= 0x1p-60f && al < 0x1p60f)
+        s->h.fast = (adaptive && c.eps >= 0x1p-100f && !(c.flags & DCASGD_RESUME)) ? kLambdaFloored : kLambdaChecked;
+    if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) s->h.fast = kLambdaLibrary; }
     s->stream = static_cast<cudaStream_t>(c.stream);
     s->device = dev;
     s->t = 0;
     s->launches = 0;
+    s->debug_status = nullptr;
+#ifdef DCASGD_DEBUG_CHECKS
+    s->debug_status = g_default_debug_status;
+#endif
     // Two vectors per thread (3 CTAs/SM, 3-stage ring) measured 4-6 % faster on B200 than one vector
     // per thread (4 CTAs/SM, 5-stage ring) once the vector is long enough to fill the GPU with
     // the larger CTAs (the per-push control work is shared by 8 elements); short vectors keep one
@@ -366,6 +422,9 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     if (const char* v = std::getenv("DCASGD_WINDOW_SLOTS")) { const int k = std::atoi(v); if (k >= 1 && k <= DCASGD_MAX_WINDOW_SLOTS) s->slot_cap = (uint32_t)k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
         // Algorithm 2, Initialize: every backup starts as w_0; MeanSquare(0) = 0
+#ifdef DCASGD_DEBUG_CHECKS
+        if (const int rc = debug_arm(s->stream, &s->cfg, s->debug_status, nullptr, 0, false)) { delete s; return rc; }
+#endif
         k_init<<<blocks_for(c.n, 1), kThreads, 0, s->stream>>>(c.w, c.w_bak, c.w_bak_stride, c.num_workers, c.ms, c.v, c.n);
         const int rc = after_launch(s, "init kernel");
         if (rc != DCASGD_OK) { delete s; return rc; }
@@ -420,6 +479,7 @@ int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, c
         }
     }
     const uint64_t gbytes = c.n * grad_elem_bytes(c);
+    uint64_t pool_extent = 0;
     if (any_push && c.n) {
         if (!grad_pool) return fail(DCASGD_EINVAL, "dcasgd_apply_log: grad_pool is NULL");
         if (!aligned16(grad_pool) || grad_stride_bytes % 16) return fail(DCASGD_EALIGN, "dcasgd_apply_log: grad_pool and grad_stride_bytes must be multiples of 16 bytes");
@@ -427,6 +487,7 @@ int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, c
         const uint64_t pool_bytes = (uint64_t)(num_grads - 1) * grad_stride_bytes + gbytes;
         if ((rc = check_foreign(c, grad_pool, pool_bytes, "grad_pool"))) return rc;
         if ((rc = check_device_buffer("dcasgd_apply_log", "grad_pool", grad_pool, pool_bytes, s->device))) return rc;
+        pool_extent = pool_bytes;
     }
 
     if (window_k == 1) {
@@ -444,7 +505,7 @@ int dcasgd_apply_log(dcasgd_server* s, const dcasgd_event* ev, uint64_t count, c
         uint64_t r = 0;
         while (r < count) {
             if ((rc = wc.compile(ev + r, count - r, window_k, c.eta, s->slot_cap, &wp))) return rc;
-            if ((rc = launch_window(s, wp, grad_pool, grad_stride_bytes))) return rc;
+            if ((rc = launch_window(s, wp, grad_pool, grad_stride_bytes, pool_extent))) return rc;
             r += wp.n_records;
         }
     } catch (const std::bad_alloc&) {
@@ -487,6 +548,9 @@ int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, voi
     uint32_t b0, b1;
     std::memcpy(&b0, &s_first, 4);
     std::memcpy(&b1, &s_last, 4);
+#ifdef DCASGD_DEBUG_CHECKS
+    if (const int rc = debug_arm(static_cast<cudaStream_t>(stream), nullptr, g_default_debug_status, mismatches_dev, 8, true)) return rc;
+#endif
     k_check_lambda<<<(unsigned)sms * 8, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         lambda0, b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
     e = cudaGetLastError();
@@ -498,6 +562,25 @@ int dcasgd_get_window_slot_cap(const dcasgd_server* s, uint32_t* max_slots) {
     if (!s || !max_slots) return fail(DCASGD_EINVAL, "dcasgd_get_window_slot_cap: NULL argument");
     *max_slots = s->slot_cap;
     return DCASGD_OK;
+}
+
+int dcasgd_debug_checks(dcasgd_server* s, uint32_t* status_dev) {
+#ifdef DCASGD_DEBUG_CHECKS
+    if (status_dev) {
+        if (reinterpret_cast<uintptr_t>(status_dev) & 3u) return fail(DCASGD_EALIGN, "dcasgd_debug_checks: status_dev must be 4-byte aligned");
+        int dev = -1;
+        const cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return cuda_fail("dcasgd_debug_checks: cudaGetDevice", e);
+        if (const int rc = check_device_buffer("dcasgd_debug_checks", "status_dev", status_dev, 4, dev)) return rc;
+    }
+    if (s) s->debug_status = status_dev;
+    else g_default_debug_status = status_dev;
+    return DCASGD_OK;
+#else
+    (void)s;
+    (void)status_dev;
+    return fail(DCASGD_EINVAL, "dcasgd_debug_checks: this library was built without -DDCASGD_DEBUG_CHECKS");
+#endif
 }
 
 int dcasgd_get_launch_count(const dcasgd_server* s, uint64_t* launches) {
