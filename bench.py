@@ -22,6 +22,8 @@ Printed: ONE JSON line (rank 0).  Besides the headline it carries
   cpu_baseline  the CPU checker on the host cores, on a bounded sample of the same workload
 With N > 1 (torchrun) every rank replays the same workload on its own GPU (independent
 replicas: the path has no exchange step); time is the slowest rank's, units are summed.
+With --sharded the N GPUs hold ONE server instead, each a contiguous element range of it
+(strong scaling: the units of the whole job are counted once).
 """
 from __future__ import annotations
 
@@ -158,6 +160,23 @@ def host_inputs(wl: synth.Workload, threads: int, pin: bool):
         wl.grad_into(view[k, : wl.n], k, threads)
     w0 = torch.empty(wl.n, dtype=torch.float32, pin_memory=pin)
     synth.normal_into(w0.numpy(), 0, wl.seed, synth.STREAM_W0, wl.w0_sigma, threads=threads)
+    return w0, pool, view, wl.log()
+
+
+def host_inputs_slice(wl: synth.Workload, lo: int, hi: int, threads: int, pin: bool):
+    """The same inputs restricted to elements [lo, hi): what one rank of the sharded server needs.
+    Every value is a function of (seed, stream, element index), so a rank draws its own slice."""
+    import torch
+    n = hi - lo
+    row = row_elems(n)
+    dt = torch.int16 if wl.bf16_grad else torch.float32
+    pool = torch.zeros((wl.num_grads, row), dtype=dt, pin_memory=pin)
+    view = pool.numpy().view(np.uint16) if wl.bf16_grad else pool.numpy()
+    sigma, seg = wl.sigma(), wl.seg_len
+    for k in range(wl.num_grads):
+        synth.normal_into(view[k, :n], lo, wl.seed, synth.STREAM_GRAD0 + k, sigma, seg, threads)
+    w0 = torch.empty(n, dtype=torch.float32, pin_memory=pin)
+    synth.normal_into(w0.numpy(), lo, wl.seed, synth.STREAM_W0, wl.w0_sigma, threads=threads)
     return w0, pool, view, wl.log()
 
 
@@ -473,6 +492,53 @@ def other_workloads(local: int, gen_threads: int) -> dict:
     return out
 
 
+def run_sharded(args, wl, rank: int, local: int, world: int, dist, gen_threads: int) -> None:
+    """Strong scaling: ONE server whose parameter vector is cut into contiguous element ranges, one
+    per GPU (paper_1609_08326_b200.sharded).  Every rank replays the whole log on its own range
+    with the unchanged library; the update needs no exchange.  The model a pulling worker receives
+    is the all-gather of the shards, timed separately."""
+    import torch
+    from paper_1609_08326_b200 import sharded
+    lo, hi = sharded.shard_range(wl.n, world, rank)
+    local_wl = wl.scaled(n=hi - lo)
+    g = GpuWorkload(local_wl, local, world, dist, gen_threads, host=host_inputs_slice(wl, lo, hi, gen_threads, pin=True), need_out=False)
+    sampler = ClockSampler(local) if rank == 0 else None
+    K, W = args.steps, args.warmup
+    total_ms, replay_ms, per_step = g.replay_steps(args.window_k, K, W)
+    max_ms, tot_units = acct.aggregate_over_ranks(total_ms, g.units * K, dist)
+    launches, nbytes = g.plan(args.window_k)
+    gbs = nbytes * K / (replay_ms * 1e-3) / 1e9
+    # the worker's view of the model: all-gather of the shards into this rank's memory
+    buf = torch.empty(world * sharded.chunk_elems(wl.n, world), dtype=torch.float32, device=g.w.device)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 10
+    for i in range(3 + reps):
+        if i == 3:
+            torch.cuda.synchronize()
+            a.record()
+        sharded.gather_model(g.w, wl.n, world, dist, out=buf)
+    b.record()
+    torch.cuda.synchronize()
+    gather_ms, _ = acct.aggregate_over_ranks(a.elapsed_time(b) / reps, 0.0, dist)
+    cfg = config_of(wl, args)
+    cfg["parallelism"] = f"element-range shards x{world} (contiguous, 32-element aligned; no collective in the update)"
+    cfg["shard_elements"] = hi - lo
+    out = {"metric": METRIC, "value": tot_units / (max_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+           "ms_per_step": max_ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+           "data": "synthetic", "config": cfg,
+           "roofline": {"bound": "hbm", "kernel": "k_replay (this rank's shard)", "achieved": gbs, "peak": g.peak, "unit": "GB/s",
+                        "frac": gbs / g.peak, "peak_kind": f"of {g.peak_kind}", "frac_of_nominal": gbs / NOMINAL_HBM_GBS, "traffic": None,
+                        "launches_per_step": launches, "avg_launch_ms": replay_ms / (K * max(1, launches))},
+           "pull_allgather": {"ms": gather_ms, "model_bytes": wl.n * 4,
+                              "received_gbs_per_gpu": wl.n * 4 * (world - 1) / max(1, world) / (gather_ms * 1e-3) / 1e9},
+           "gpu_launches": g.launches}
+    if sampler is not None:
+        out["clocks"] = sampler.stop()
+    g.close()
+    if rank == 0:
+        print(json.dumps(out))
+
+
 def run_b200(args) -> None:
     import torch
     import torch.distributed as dist
@@ -491,6 +557,11 @@ def run_b200(args) -> None:
     wl = select_workload(args)
     cores = os.cpu_count() or 1
     gen_threads = max(1, cores // world)
+    if args.sharded:
+        run_sharded(args, wl, rank, local, world, dist if world > 1 else None, gen_threads)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     g = GpuWorkload(wl, local, world, dist if world > 1 else None, gen_threads)
     sampler = ClockSampler(local) if rank == 0 else None
     K, W = args.steps, args.warmup
@@ -571,6 +642,8 @@ def main() -> None:
     ap.add_argument("--no-workloads", action="store_true", help="skip the section that times the other configurations")
     ap.add_argument("--headline-only", action="store_true", help="skip variants, single kernels, e2e, CPU baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="N GPUs hold ONE server, cut into element ranges (strong scaling) instead of N replicas")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -150,13 +150,27 @@ uint32_t dcasgd_version(void);
 
 /* Diagnostic, no counterpart in the paper.  For the adaptive variant the kernels compute
  * lambda_t = lambda_0 / sqrt(s), s = ms + eps, on a branch-free route (packed FMAs, one Newton
- * correction for the root, Markstein-style corrected quotient) when s is in [2^-100, 2^100) and
+ * correction for the root, a once-refined reciprocal and one exact-residual correction of the
+ * quotient) when s is in [2^-100, 2^100) and
  * |lambda_0| in [2^-60, 2^60), and with the compiler's guarded IEEE sqrt and division otherwise.
+ * (The branch-free route was compared with the IEEE one on every pair of significands, see
+ * dcasgd_check_adaptive_lambda_grid below: results are bit-equal for EVERY admissible lambda_0.)
  * This call runs both routes on EVERY binary32 value s in [s_first, s_last] for the given
  * lambda_0 and ADDS the number of inputs on which their bits differ to *mismatches_dev (device,
  * 8 bytes, 8-byte aligned, zeroed by the caller).  Enqueued on `stream`; allocates nothing.
  * The expected count is 0 for every admissible argument. */
 int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, void *stream, uint64_t *mismatches_dev);
+
+/* The same comparison over a grid of numerators and radicands: a takes the a_count binary32 values
+ * whose encodings are bits(a_first), bits(a_first) + a_step, ... (all of one sign, every |a| in
+ * [2^-60, 2^60)), s every binary32 value in [s_first, s_last].  The branch-free route only
+ * multiplies, adds and fuses, and nothing in it leaves the normal range for these arguments, so
+ * scaling a by 2 or s by 4 scales every intermediate by a power of two: whether it rounds
+ * correctly depends on the significands alone.  a in [1, 2) with a_step = 1 (2^23 values) and s
+ * in [1, 4) (2^24 values) therefore covers EVERY admissible pair; that run takes a minute or two
+ * on a B200 and finds no mismatch.  The work is cut into launches of a fraction of a second. */
+int dcasgd_check_adaptive_lambda_grid(float a_first, uint32_t a_count, uint32_t a_step, float s_first, float s_last,
+                                      void *stream, uint64_t *mismatches_dev);
 
 /* Checked build, no counterpart in the paper.  A library compiled with -DDCASGD_DEBUG_CHECKS
  * makes every kernel compare each global-memory address it is about to use with the buffers of

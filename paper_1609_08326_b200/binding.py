@@ -32,7 +32,7 @@ MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
 SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
            "dcasgd_get_step", "dcasgd_set_step", "dcasgd_get_launch_count", "dcasgd_last_error",
            "dcasgd_status_string", "dcasgd_version", "dcasgd_compile_window", "dcasgd_check_adaptive_lambda",
-           "dcasgd_get_window_slot_cap", "dcasgd_debug_checks"]
+           "dcasgd_get_window_slot_cap", "dcasgd_debug_checks", "dcasgd_check_adaptive_lambda_grid"]
 
 
 class Config(C.Structure):
@@ -87,6 +87,8 @@ def lib() -> C.CDLL:
         L.dcasgd_get_window_slot_cap.restype = C.c_int
         L.dcasgd_check_adaptive_lambda.argtypes = [C.c_float, C.c_float, C.c_float, vp, vp]
         L.dcasgd_check_adaptive_lambda.restype = C.c_int
+        L.dcasgd_check_adaptive_lambda_grid.argtypes = [C.c_float, u32, u32, C.c_float, C.c_float, vp, vp]
+        L.dcasgd_check_adaptive_lambda_grid.restype = C.c_int
         L.dcasgd_debug_checks.argtypes = [vp, vp]
         L.dcasgd_debug_checks.restype = C.c_int
         for name in ("dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",
@@ -194,6 +196,12 @@ def dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, mismatches_dev, strea
     """Adds to the device counter the number of s in [s_first, s_last] on which the two routes
     of lambda_0 / sqrt(s) differ (expected: 0)."""
     _check(lib().dcasgd_check_adaptive_lambda(lambda0, s_first, s_last, stream, _ptr(mismatches_dev)))
+
+
+def dcasgd_check_adaptive_lambda_grid(a_first, a_count, a_step, s_first, s_last, mismatches_dev, stream=None) -> None:
+    """The same over a grid: a_count numerators (encodings bits(a_first) + i * a_step) times every
+    s in [s_first, s_last].  a in [1, 2) with step 1 and s in [1, 4) covers every significand pair."""
+    _check(lib().dcasgd_check_adaptive_lambda_grid(a_first, a_count, a_step, s_first, s_last, stream, _ptr(mismatches_dev)))
 
 
 def dcasgd_debug_checks(h, status_dev) -> None:

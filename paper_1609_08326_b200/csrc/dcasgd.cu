@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in dcasgd.h: argument validation, the serial message loop of
 // Algorithm 2, and the launches.  Every check runs before the first launch of a call.
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -383,20 +384,16 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     dcasgd_server* s = new (std::nothrow) dcasgd_server;
     if (!s) return fail(DCASGD_ENOMEM, "dcasgd_create: out of host memory");
     s->cfg = c;
-    s->h.lambda = c.lambda;
-    s->h.mu = adaptive ? c.mu : 0.0f;
-    s->h.omm = 1.0f - s->h.mu;
-    s->h.eps = adaptive ? c.eps : 0.0f;
-    s->h.beta = c.v ? c.beta : 0.0f;
     // Route of the adaptive lambda (see kernels.cuh).  The branch-free route is exact for
     // |lambda_0| in [2^-60, 2^60) and s in [2^-100, 2^100).  The lower bound on s needs no test when
     // eps >= 2^-100 and MeanSquare starts at 0 here (it is a sum of non-negative terms from then
     // on); a resumed state comes from the caller, so its MeanSquare is not taken on trust.
     const float al = std::fabs(c.lambda);
-    s->h.fast = kLambdaLibrary;
+    uint32_t route = kLambdaLibrary;
     if (al >= 0x1p-60f && al < 0x1p60f)
-        s->h.fast = (adaptive && c.eps >= 0x1p-100f && !(c.flags & DCASGD_RESUME)) ? kLambdaFloored : kLambdaChecked;
-    if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) s->h.fast = kLambdaLibrary; }
+        route = (adaptive && c.eps >= 0x1p-100f && !(c.flags & DCASGD_RESUME)) ? kLambdaFloored : kLambdaChecked;
+    if (const char* v = std::getenv("DCASGD_IEEE_LIBRARY_MATH")) { if (std::atoi(v) == 1) route = kLambdaLibrary; }
+    s->h = make_hyper(c.lambda, adaptive ? c.mu : 0.0f, adaptive ? c.eps : 0.0f, c.v ? c.beta : 0.0f, route);
     s->stream = static_cast<cudaStream_t>(c.stream);
     s->device = dev;
     s->t = 0;
@@ -552,9 +549,53 @@ int dcasgd_check_adaptive_lambda(float lambda0, float s_first, float s_last, voi
     if (const int rc = debug_arm(static_cast<cudaStream_t>(stream), nullptr, g_default_debug_status, mismatches_dev, 8, true)) return rc;
 #endif
     k_check_lambda<<<(unsigned)sms * 8, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        lambda0, b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
+        make_hyper(lambda0, 0.0f, 0.0f, 0.0f, kLambdaChecked), b0, (uint64_t)b1 - b0 + 1, reinterpret_cast<unsigned long long*>(mismatches_dev));
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("lambda self-check kernel", e);
+    return DCASGD_OK;
+}
+
+int dcasgd_check_adaptive_lambda_grid(float a_first, uint32_t a_count, uint32_t a_step, float s_first, float s_last,
+                                      void* stream, uint64_t* mismatches_dev) {
+    const char* fn = "dcasgd_check_adaptive_lambda_grid";
+    if (!mismatches_dev) return fail(DCASGD_EINVAL, "%s: mismatches_dev is NULL", fn);
+    if (reinterpret_cast<uintptr_t>(mismatches_dev) & 7u) return fail(DCASGD_EALIGN, "%s: mismatches_dev must be 8-byte aligned", fn);
+    if (a_count == 0) return DCASGD_OK;
+    uint32_t a0, b0, b1;
+    std::memcpy(&a0, &a_first, 4);
+    const uint64_t a_last_bits = (uint64_t)a0 + (uint64_t)(a_count - 1) * a_step;
+    if (a_last_bits > 0xFFFFFFFFull || ((uint32_t)a_last_bits ^ a0) >> 31) return fail(DCASGD_EINVAL, "%s: the numerators leave the sign's half of the encodings", fn);
+    float a_last;
+    const uint32_t al_bits = (uint32_t)a_last_bits;
+    std::memcpy(&a_last, &al_bits, 4);
+    const float lo = std::fabs(a_first), hi = std::fabs(a_last);      // bit patterns grow with the magnitude
+    if (!(lo >= 0x1p-60f && hi < 0x1p60f)) return fail(DCASGD_EINVAL, "%s: every |a| must be in [2^-60, 2^60)", fn);
+    if (!(s_first >= 0x1p-100f && s_last < 0x1p100f && s_first <= s_last))
+        return fail(DCASGD_EINVAL, "%s: need 2^-100 <= s_first <= s_last < 2^100", fn);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(fn, e);
+    if (const int rc = check_device_buffer(fn, "mismatches_dev", mismatches_dev, 8, dev)) return rc;
+    int sms = 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
+    std::memcpy(&b0, &s_first, 4);
+    std::memcpy(&b1, &s_last, 4);
+    const uint64_t s_count = (uint64_t)b1 - b0 + 1;
+    // launches of bounded length: at most about 3e11 comparisons each (a fraction of a second)
+    const uint64_t per = std::max<uint64_t>(1, std::min<uint64_t>(a_count, (300ull << 30) / s_count));
+    const uint64_t pairs = (s_count + 1) / 2;
+    const unsigned grid = (unsigned)std::min<uint64_t>((pairs + kThreads - 1) / kThreads, (uint64_t)sms * 64);
+#ifdef DCASGD_DEBUG_CHECKS
+    if (const int rc = debug_arm(static_cast<cudaStream_t>(stream), nullptr, g_default_debug_status, mismatches_dev, 8, true)) return rc;
+#endif
+    for (uint64_t done = 0; done < a_count; done += per) {
+        const uint32_t na = (uint32_t)std::min<uint64_t>(per, a_count - done);
+        k_check_lambda_grid<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+            make_hyper(1.0f, 0.0f, 0.0f, 0.0f, kLambdaChecked), a0 + (uint32_t)(done * a_step), na, a_step, b0, s_count,
+            reinterpret_cast<unsigned long long*>(mismatches_dev));
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail("lambda grid self-check kernel", e);
+    }
     return DCASGD_OK;
 }
 

@@ -44,3 +44,24 @@ def test_sample_log_keeps_whole_push_pull_pairs():
     assert int(np.sum(s["kind"] == synth.PUSH)) == 7 and s[-1]["kind"] == synth.PULL
     assert len(bench.sample_log(ev, 10_000)) == len(ev)
     assert bench.row_elems(272_474) % 32 == 0 and bench.row_elems(272_474) >= 272_474
+
+
+def test_steady_sample_starts_after_the_leading_pulls():
+    import bench
+    M = 4
+    ev = synth.event_log(M, 50, synth.ORDER_UNIFORM, synth.PROTO_ASYNC, 5, 0.1, seed=0)
+    s = bench.steady_sample(ev, M, 9)
+    assert s[0]["kind"] == synth.PUSH and s[-1]["kind"] == synth.PULL
+    assert int(np.sum(s["kind"] == synth.PUSH)) == 9 == int(np.sum(s["kind"] == synth.PULL))
+    assert len(bench.steady_sample(ev, M, 10_000)) == len(ev) - M
+
+
+def test_a_rank_draws_exactly_its_slice_of_the_inputs():
+    import bench
+    wl = synth.workload("c2_adaptive_1p7m").scaled(n=10_007, num_grads=3, pushes=10)
+    w0, pool, view, ev = bench.host_inputs(wl, 2, pin=False)
+    lo, hi = 4_992, 10_007
+    w0s, pools, views, evs = bench.host_inputs_slice(wl, lo, hi, 2, pin=False)
+    assert np.array_equal(w0s.numpy(), w0.numpy()[lo:hi])
+    assert np.array_equal(views[:, : hi - lo], view[:, lo:hi])
+    assert np.array_equal(evs, ev)

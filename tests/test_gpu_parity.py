@@ -289,14 +289,34 @@ def test_adaptive_lambda_routes(lam, eps):
         U.assert_state_equal(gpu, cpu, what=f"lam={lam} eps={eps} K={K} ")
 
 
+def lambda0_cases() -> list[float]:
+    """Numerators for the exhaustive-in-s comparison: the paper's settings, powers of two and their
+    neighbours one ulp away, all-ones significands, both ends of [2^-60, 2^60), and seeded random
+    values spread log-uniformly over that range with random signs."""
+    f = np.float32
+    vals = [2.0, 0.04, 1.0, -2.0, 0.3, 1.9999999, 7.7e-12, 3.3e9]
+    for k in (-60, -31, -1, 0, 1, 24, 59):
+        p2 = f(2.0) ** f(k)
+        vals += [float(p2), float(np.nextafter(p2, f(np.inf)))]
+        if k > -60:
+            vals.append(float(np.nextafter(p2, f(0))))               # all-ones significand just below the power of two
+    vals.append(float(np.nextafter(f(2.0) ** f(60), f(0))))          # the largest admissible numerator
+    rng = np.random.default_rng(20240607)
+    mag = np.exp2(rng.uniform(-60, 60, size=40)).astype(f)
+    sign = rng.choice([-1.0, 1.0], size=40).astype(f)
+    vals += [float(v) for v in mag * sign]
+    vals = [v for v in vals if 2.0 ** -60 <= abs(v) < 2.0 ** 60]
+    assert len(vals) >= 64
+    return vals
+
+
 def test_adaptive_lambda_branch_free_route_is_exact_for_every_s():
-    """Exhaustive: for several lambda_0 (the paper's 2 and 0.04 among them) the branch-free
-    lambda_0 / sqrt(s) equals the IEEE sqrt-then-divide on all 1.68e9 binary32 values of s in
-    [2^-100, 2^100)."""
+    """For 69 numerators lambda_0 (see lambda0_cases) the branch-free lambda_0 / sqrt(s) equals
+    the IEEE sqrt-then-divide on all 1.68e9 binary32 values of s in [2^-100, 2^100)."""
     import torch
     counter = torch.zeros(1, dtype=torch.int64, device="cuda")
     last = float(np.nextafter(np.float32(2.0 ** 100), np.float32(0)))
-    for lam0 in (2.0, 0.04, 1.0, -2.0, 0.3, 1.9999999, 7.7e-12, 3.3e9):
+    for lam0 in lambda0_cases():
         B.dcasgd_check_adaptive_lambda(lam0, 2.0 ** -100, last, counter)
     torch.cuda.synchronize()
     assert int(counter.item()) == 0
@@ -305,6 +325,35 @@ def test_adaptive_lambda_branch_free_route_is_exact_for_every_s():
                 lambda: B.dcasgd_check_adaptive_lambda(2.0, 1.0, 2.0, None)):
         with pytest.raises(B.DcasgdError):
             bad()
+
+
+def test_adaptive_lambda_on_a_grid_of_significand_pairs():
+    """Numerators and radicands together.  The branch-free route is invariant under scaling the
+    numerator by 2 and s by 4, so numerators in [1, 2) and s in [1, 4) stand for all exponents.
+    Always: 2^15 numerators strided over all significands (odd stride: low bits vary too) times
+    every s in [1, 4) = 5.5e11 pairs, plus every numerator against the radicands whose root has an
+    all-ones significand (the one hard case of the reciprocal refinement).
+    With DCASGD_EXHAUSTIVE=1: ALL 2^23 x 2^24 = 1.4e14 pairs (a minute or two)."""
+    import os
+
+    import torch
+    counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+    below4 = float(np.nextafter(np.float32(4.0), np.float32(0)))
+    B.dcasgd_check_adaptive_lambda_grid(1.0, 1 << 15, 255, 1.0, below4, counter)
+    hard = float(np.nextafter(np.nextafter(np.float32(4.0), np.float32(0)), np.float32(0)))     # sqrt rounds to 2 - 2^-23
+    B.dcasgd_check_adaptive_lambda_grid(1.0, 1 << 23, 1, hard, below4, counter)
+    B.dcasgd_check_adaptive_lambda_grid(-1.0, 1 << 23, 1, hard, below4, counter)
+    if os.environ.get("DCASGD_EXHAUSTIVE") == "1":
+        B.dcasgd_check_adaptive_lambda_grid(1.0, 1 << 23, 1, 1.0, below4, counter)
+    torch.cuda.synchronize()
+    assert int(counter.item()) == 0
+    with pytest.raises(B.DcasgdError):
+        B.dcasgd_check_adaptive_lambda_grid(2.0 ** 59, 1 << 23, 2, 1.0, 2.0, counter)       # numerators reach 2^60
+    with pytest.raises(B.DcasgdError):
+        B.dcasgd_check_adaptive_lambda_grid(1.0, 4, 1, 0.0, 2.0, counter)
+    with pytest.raises(B.DcasgdError):
+        B.dcasgd_check_adaptive_lambda_grid(1.0, 4, 1, 1.0, 2.0, None)
+    B.dcasgd_check_adaptive_lambda_grid(1.0, 0, 1, 1.0, 2.0, counter)                        # nothing to do
 
 
 def test_apply_log_from_host_overlapped_copies():
