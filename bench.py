@@ -461,8 +461,8 @@ class GpuWorkload:
 # the other configurations of the benchmark set, each with a step count of its own (independent of
 # --steps) sized so that the whole section takes about a minute: (timed steps, window sizes)
 OTHER_WORKLOADS = {
-    "c1_resnet20_const": (20, (32, 8, 256, 1)),
-    "c2_adaptive_1p7m": (6, (32, 8, 256, 1)),
+    "c1_resnet20_const": (20, (32, 8, 256, 1280, 1)),
+    "c2_adaptive_1p7m": (6, (32, 8, 256, 1280, 1)),
     "c4_vgg16_const_bf16": (2, (32, 8, 1)),
     "c4_vgg16_adaptive_bf16": (2, (32, 8, 1)),
 }

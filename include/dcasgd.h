@@ -199,9 +199,12 @@ int dcasgd_debug_checks(dcasgd_server *s, uint32_t *status_dev);
  *                     superseded inside the window without being used cost nothing.
  * The window is shortened (n_records < window_k) when it would need more than
  * max_slots (at most DCASGD_MAX_WINDOW_SLOTS) live snapshots, DCASGD_MAX_WINDOW_PUSHES pushes or
- * DCASGD_MAX_WINDOW_STORES stores; the remaining records start the next window. */
-#define DCASGD_MAX_WINDOW_PUSHES 128
-#define DCASGD_MAX_WINDOW_STORES 192
+ * DCASGD_MAX_WINDOW_STORES stores; the remaining records start the next window.  (The program
+ * travels to the kernel as a launch parameter: a window of up to 128 pushes and 192 stores in
+ * a 5.6 KB form, a longer one in a 28 KB form.  Long windows pay off where the vector is short
+ * and a launch would otherwise cost as much as the work it carries.) */
+#define DCASGD_MAX_WINDOW_PUSHES 640
+#define DCASGD_MAX_WINDOW_STORES 960
 #define DCASGD_MAX_WINDOW_SLOTS 16
 
 typedef struct {

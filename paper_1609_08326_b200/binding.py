@@ -26,7 +26,7 @@ CONST, ADAPTIVE = 0, 1
 F32, BF16 = 0, 1
 PULL, PUSH = 0, 1
 RESUME = 1
-MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 128, 192, 16
+MAX_WINDOW_PUSHES, MAX_WINDOW_STORES, MAX_WINDOW_SLOTS = 640, 960, 16
 
 # every symbol include/dcasgd.h declares
 SYMBOLS = ["dcasgd_create", "dcasgd_pull", "dcasgd_push", "dcasgd_apply_log", "dcasgd_destroy",

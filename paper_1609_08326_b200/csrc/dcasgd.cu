@@ -19,6 +19,7 @@ struct dcasgd_server {
     Hyper h;
     cudaStream_t stream;
     int device;
+    int sms;             // multiprocessors of the device
     int replay_vecs;     // 16-byte vectors per thread in the fused replay kernel (1 or 2) for windows with few slots
     uint32_t two_vec_slots;  // a window that needs more slots than this runs one vector per thread
     uint32_t slot_cap;   // in-window snapshot slots a window may use
@@ -220,17 +221,14 @@ int launch_push(dcasgd_server* s, uint32_t m, const void* g, float eta) {
     return rc;
 }
 
-int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void* grad_pool,
-                  uint64_t grad_stride_bytes, uint64_t pool_bytes) {
-    const dcasgd_config& c = s->cfg;
-    if (c.n == 0) { s->t += wp.n_pushes; return DCASGD_OK; }
-    if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
-    // many live snapshots: one vector per thread keeps two CTAs per SM resident (a slot costs half)
-    const int V = wp.n_slots > s->two_vec_slots ? 1 : s->replay_vecs;
+// Fills the device form of a window program: everything a thread would otherwise compute per
+// push is resolved here (byte offsets in the pool and in w_bak, shared-memory offsets of the
+// snapshot a push reads and of the slot that keeps w after it).
+template <class PROG>
+void fill_program(PROG& p, const dcasgd_window_program& wp, const dcasgd_config& c, uint64_t grad_stride_bytes, int V) {
     const int S = replay_stages(V);
-    static thread_local DevProgram p;            // 5.6 KB: kept off the stack
-    std::memset(&p, 0, sizeof p);
     p.n_pushes = wp.n_pushes;
+    p.pad = 0;
     p.save_off0 = wp.save_slot[0] >= 0 ? replay_slot_off(V, (uint32_t)wp.save_slot[0]) : kNoSave;
     p.store_end0 = wp.store_begin[1];
     for (uint32_t j = 0; j < wp.n_pushes; ++j) {
@@ -249,6 +247,36 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
         ap.store_end = wp.store_begin[j + 2];
     }
     for (uint32_t k = 0; k < wp.n_stores; ++k) p.store_off[k] = (uint64_t)wp.store_worker[k] * c.w_bak_stride * 4;
+}
+
+template <class PROG>
+void launch_replay(const dcasgd_server* s, const ReplayArgs& a, const PROG& p, int V, unsigned grid, size_t smem) {
+    const dcasgd_config& c = s->cfg;
+    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
+#define DCASGD_LAUNCH_REPLAY(AD, BF)                                                               \
+    do {                                                                                           \
+        if (mom) {                                                                                 \
+            if (V == 2) k_replay<AD, BF, true, 2, PROG><<<grid, kThreads, smem, s->stream>>>(a, p);  \
+            else        k_replay<AD, BF, true, 1, PROG><<<grid, kThreads, smem, s->stream>>>(a, p);  \
+        } else {                                                                                   \
+            if (V == 2) k_replay<AD, BF, false, 2, PROG><<<grid, kThreads, smem, s->stream>>>(a, p); \
+            else        k_replay<AD, BF, false, 1, PROG><<<grid, kThreads, smem, s->stream>>>(a, p); \
+        }                                                                                          \
+    } while (0)
+    if (ad && bf)       DCASGD_LAUNCH_REPLAY(true, true);
+    else if (ad)        DCASGD_LAUNCH_REPLAY(true, false);
+    else if (bf)        DCASGD_LAUNCH_REPLAY(false, true);
+    else                DCASGD_LAUNCH_REPLAY(false, false);
+#undef DCASGD_LAUNCH_REPLAY
+}
+
+int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void* grad_pool,
+                  uint64_t grad_stride_bytes, uint64_t pool_bytes) {
+    const dcasgd_config& c = s->cfg;
+    if (c.n == 0) { s->t += wp.n_pushes; return DCASGD_OK; }
+    if (wp.n_pushes == 0 && wp.n_stores == 0) return DCASGD_OK;   // nothing survives this window
+    // many live snapshots: one vector per thread keeps two CTAs per SM resident (a slot costs half)
+    const int V = wp.n_slots > s->two_vec_slots ? 1 : s->replay_vecs;
     ReplayArgs a;
     a.w = c.w;
     a.w_bak = c.w_bak;
@@ -261,34 +289,32 @@ int launch_window(dcasgd_server* s, const dcasgd_window_program& wp, const void*
     const size_t smem = replay_smem_bytes(wp.n_slots, V);
     DCASGD_DEBUG_ARM(s, grad_pool, pool_bytes, false);
     (void)pool_bytes;
-    const bool ad = c.variant == DCASGD_ADAPTIVE, bf = c.grad_dtype == DCASGD_BF16, mom = c.v != nullptr;
-#define DCASGD_LAUNCH_REPLAY(AD, BF)                                                         \
-    do {                                                                                     \
-        if (mom) {                                                                           \
-            if (V == 2) k_replay<AD, BF, true, 2><<<grid, kThreads, smem, s->stream>>>(a, p); \
-            else        k_replay<AD, BF, true, 1><<<grid, kThreads, smem, s->stream>>>(a, p); \
-        } else {                                                                             \
-            if (V == 2) k_replay<AD, BF, false, 2><<<grid, kThreads, smem, s->stream>>>(a, p); \
-            else        k_replay<AD, BF, false, 1><<<grid, kThreads, smem, s->stream>>>(a, p); \
-        }                                                                                    \
-    } while (0)
-    if (ad && bf)       DCASGD_LAUNCH_REPLAY(true, true);
-    else if (ad)        DCASGD_LAUNCH_REPLAY(true, false);
-    else if (bf)        DCASGD_LAUNCH_REPLAY(false, true);
-    else                DCASGD_LAUNCH_REPLAY(false, false);
-#undef DCASGD_LAUNCH_REPLAY
+    if (wp.n_pushes <= (uint32_t)DevProgram::kPushes && wp.n_stores <= (uint32_t)DevProgram::kStores) {
+        static thread_local DevProgram p;        // kept off the stack
+        fill_program(p, wp, c, grad_stride_bytes, V);
+        launch_replay(s, a, p, V, grid, smem);
+    } else {
+        static thread_local DevProgramLong p;
+        fill_program(p, wp, c, grad_stride_bytes, V);
+        launch_replay(s, a, p, V, grid, smem);
+    }
     const int rc = after_launch(s, "window replay kernel");
     if (rc == DCASGD_OK) s->t += wp.n_pushes;
     return rc;
 }
 
-template <bool AD, bool BF, bool MOM>
-cudaError_t allow_slots_one() {
-    cudaError_t e = cudaFuncSetAttribute(k_replay<AD, BF, MOM, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <bool AD, bool BF, bool MOM, class PROG>
+cudaError_t allow_slots_prog() {
+    cudaError_t e = cudaFuncSetAttribute(k_replay<AD, BF, MOM, 1, PROG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 1));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(k_replay<AD, BF, MOM, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(k_replay<AD, BF, MOM, 2, PROG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)replay_smem_bytes(DCASGD_MAX_WINDOW_SLOTS, 2));
+}
+template <bool AD, bool BF, bool MOM>
+cudaError_t allow_slots_one() {
+    const cudaError_t e = allow_slots_prog<AD, BF, MOM, DevProgram>();
+    return e != cudaSuccess ? e : allow_slots_prog<AD, BF, MOM, DevProgramLong>();
 }
 template <bool AD, bool BF>
 cudaError_t allow_slots() {
@@ -408,6 +434,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     // vector per thread for the parallelism.  DCASGD_REPLAY_VECS=1|2 overrides the choice.
     int sms = 148;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) { (void)cudaGetLastError(); sms = 148; }
+    s->sms = sms;
     s->replay_vecs = blocks_for(c.n, 2) >= 2u * (unsigned)sms ? 2 : 1;
     if (const char* v = std::getenv("DCASGD_REPLAY_VECS")) { const int k = std::atoi(v); if (k == 1 || k == 2) s->replay_vecs = k; }
     // A slot costs 4 KB (8 KB with two vectors per thread) of shared memory per CTA on top of the

@@ -98,7 +98,7 @@ def test_record_soup_and_limits():
         slots += [(PUSH, k, k % G), (PULL, k)]
     slots += [(PUSH, k, k % G) for k in range(M)]
     logs.append(synth.make_log(slots))
-    logs.append(synth.make_log([(PUSH, 0, k % G) for k in range(300)]))
+    logs.append(synth.make_log([(PUSH, 0, k % G) for k in range(1500)]))
     logs.append(synth.make_log([(PUSH, 0, 0)] + [(PULL, m % M) for m in range(250)] + [(PUSH, 3, 1)]))
     wl = small_workload(n, True, False, M=M, G=G)
     w0, pool = wl.w0(), U.host_pool(wl)
@@ -109,6 +109,33 @@ def test_record_soup_and_limits():
             gpu.apply_log(ev, dpool, K)
             cpu.replay(ev, np.ascontiguousarray(pool[:, :n]))
             U.assert_state_equal(gpu, cpu)
+
+
+@pytest.mark.parametrize("adaptive,bf16", [(False, False), (True, True)])
+def test_long_windows_take_the_large_program(adaptive, bf16):
+    """Windows of several hundred pushes (short vectors: launches are what costs) travel in the
+    28 KB form of the window program; more pushes or stores than even that holds cut the window."""
+    wl = small_workload(3001, adaptive, bf16, M=4, pushes=1500, G=11, seed=5)
+    ev, w0, pool = wl.log(), wl.w0(), U.host_pool(wl)
+    dpool = U.to_device(pool)
+    for K in (600, 1280, 100_000):
+        gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+        gpu.apply_log(ev, dpool, K)
+        cpu.replay(ev, pool[:, : wl.n])
+        U.assert_state_equal(gpu, cpu, what=f"K={K} ")
+        progs = B.plan_log(ev, wl.M, K, wl.eta, B.dcasgd_get_window_slot_cap(gpu.h))
+        assert gpu.launches == 1 + sum(1 for p in progs if p.n_pushes or p.n_stores)
+        assert max(p.n_pushes for p in progs) == min(B.MAX_WINDOW_PUSHES, K // 2)
+    # more final pulls than a window can store: 1100 workers all pull after one push
+    M = 1100
+    wl = small_workload(64, adaptive, bf16, M=M, pushes=4, G=3)
+    w0, pool = wl.w0(), U.host_pool(wl)
+    ev = synth.make_log([(PUSH, 0, 0)] + [(PULL, m) for m in range(M)] + [(PUSH, 3, 1), (PULL, 7), (PUSH, 1099, 2)])
+    gpu, cpu = U.gpu_server(wl, w0), U.cpu_server(wl, w0)
+    gpu.apply_log(ev, U.to_device(pool), 100_000)
+    cpu.replay(ev, pool[:, : wl.n])
+    U.assert_state_equal(gpu, cpu)
+    assert gpu.launches == 3
 
 
 def test_apply_log_in_pieces_and_step_counter():

@@ -132,12 +132,12 @@ def test_limits_cut_the_window():
     progs = check(ev, M, 1000, G=5)
     assert len(progs) > 1 and max(p.n_slots for p in progs) == B.MAX_WINDOW_SLOTS
     # more pushes than a window holds
-    ev = synth.make_log([(PUSH, 0, k % 5) for k in range(300)])
-    progs = check(ev, 1, 1000, G=5)
-    assert [p.n_pushes for p in progs] == [128, 128, 44]
+    ev = synth.make_log([(PUSH, 0, k % 5) for k in range(1500)])
+    progs = check(ev, 1, 1_000_000, G=5)
+    assert [p.n_pushes for p in progs] == [B.MAX_WINDOW_PUSHES, B.MAX_WINDOW_PUSHES, 1500 - 2 * B.MAX_WINDOW_PUSHES]
     # more final pulls than a window can store
-    ev = synth.make_log([(PUSH, 0, 0)] + [(PULL, m) for m in range(250)] + [(PUSH, 3, 1)])
-    progs = check(ev, 250, 1000, G=5)
+    ev = synth.make_log([(PUSH, 0, 0)] + [(PULL, m) for m in range(1100)] + [(PUSH, 3, 1)])
+    progs = check(ev, 1100, 1_000_000, G=5)
     assert progs[0].n_stores == B.MAX_WINDOW_STORES and len(progs) == 2
 
 
