@@ -43,6 +43,11 @@
  *   Threads    One server handle is used by one host thread at a time.
  *   Legal      A push with no earlier pull (the backup still holds w_0), repeated pushes on one
  *              pull, repeated pulls: Algorithm 2 has no rule against them, neither has this.
+ *   Tuning     Read by dcasgd_create from the environment; none changes a result, only speed.
+ *              DCASGD_REPLAY_VECS=1|2      16-byte vectors per thread in the fused kernel
+ *              DCASGD_TWO_VEC_SLOTS=k      windows with more than k live snapshots run one vector per thread (default 8)
+ *              DCASGD_WINDOW_SLOTS=k       live snapshots a window may keep before it is cut (default 16)
+ *              DCASGD_IEEE_LIBRARY_MATH=1  adaptive lambda always through the compiler's sqrt and division
  */
 #ifndef DCASGD_H
 #define DCASGD_H

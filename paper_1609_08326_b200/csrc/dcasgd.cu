@@ -442,6 +442,7 @@ int dcasgd_create(const dcasgd_config* cfg, dcasgd_server** out) {
     // SM); longer windows over many workers need up to 16 and run one vector per thread (2 CTAs
     // per SM), which measured faster than cutting them at 8 slots.
     s->two_vec_slots = 8;
+    if (const char* v = std::getenv("DCASGD_TWO_VEC_SLOTS")) { const int k = std::atoi(v); if (k >= 0 && k <= DCASGD_MAX_WINDOW_SLOTS) s->two_vec_slots = (uint32_t)k; }
     s->slot_cap = DCASGD_MAX_WINDOW_SLOTS;
     if (const char* v = std::getenv("DCASGD_WINDOW_SLOTS")) { const int k = std::atoi(v); if (k >= 1 && k <= DCASGD_MAX_WINDOW_SLOTS) s->slot_cap = (uint32_t)k; }
     if (c.n && !(c.flags & DCASGD_RESUME)) {
@@ -612,12 +613,14 @@ int dcasgd_check_adaptive_lambda_grid(float a_first, uint32_t a_count, uint32_t 
     const uint64_t per = std::max<uint64_t>(1, std::min<uint64_t>(a_count, (300ull << 30) / s_count));
     const uint64_t pairs = (s_count + 1) / 2;
     const unsigned grid = (unsigned)std::min<uint64_t>((pairs + kThreads - 1) / kThreads, (uint64_t)sms * 64);
+    // few radicands: spread the numerators over blockIdx.y until the GPU is full
+    const unsigned grid_y = (unsigned)std::max<uint64_t>(1, std::min<uint64_t>({(uint64_t)sms * 8 / grid, (uint64_t)per, 4096}));
 #ifdef DCASGD_DEBUG_CHECKS
     if (const int rc = debug_arm(static_cast<cudaStream_t>(stream), nullptr, g_default_debug_status, mismatches_dev, 8, true)) return rc;
 #endif
     for (uint64_t done = 0; done < a_count; done += per) {
         const uint32_t na = (uint32_t)std::min<uint64_t>(per, a_count - done);
-        k_check_lambda_grid<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        k_check_lambda_grid<<<dim3(grid, grid_y), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
             make_hyper(1.0f, 0.0f, 0.0f, 0.0f, kLambdaChecked), a0 + (uint32_t)(done * a_step), na, a_step, b0, s_count,
             reinterpret_cast<unsigned long long*>(mismatches_dev));
         e = cudaGetLastError();
