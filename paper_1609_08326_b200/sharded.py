@@ -80,10 +80,13 @@ def scatter_gradient(full, n: int, world: int, rank: int, src: int, dist=None, g
     if dist is None or world == 1:
         return full[lo:hi]
     if out is None:
-        ref = full if full is not None else None
-        if ref is None:
+        if full is None:
             raise ValueError("ranks other than src must pass a receive buffer `out`")
-        out = torch.empty(c, dtype=ref.dtype, device=ref.device)
+        out = torch.empty(c, dtype=full.dtype, device=full.device)
+    if out.numel() != c:
+        raise ValueError("the receive buffer must hold chunk_elems(n, world) elements")
+    if rank == src and (full is None or full.numel() < n):
+        raise ValueError("rank src must pass the full gradient (n elements)")
     pieces = None
     if rank == src:
         padded = full
