@@ -1,5 +1,6 @@
 """GPU parity at the full sizes of the benchmark workloads, in the launch configurations that
-bench.py times (fused windows of 32 and 8 records, and one kernel per message).
+bench.py times (fused windows of 8, 32 and 256 records, 1280 records on the short vectors, and
+one kernel per message).
 
 The CPU checker replays the FULL log on a sample of elements (head and tail of the vector, the
 neighbourhood of every gradient-scale segment boundary, and a regular stride): elements never
@@ -36,7 +37,7 @@ def test_c1_resnet20_constant_full_vector_full_log():
     assert len(ev) == 4 + 2 * 2000 and pool.shape[0] == 2000
     dpool = U.to_device(pool)
     servers, bounds = U.cpu_replay_ranges(wl, ev, w0, pool, os.cpu_count() or 1)
-    for K in (32, 8, 1):
+    for K in (32, 8, 256, 1280, 1):
         gpu = U.gpu_server(wl, w0)
         gpu.apply_log(ev, dpool, K)
         U.assert_ranges_equal(gpu, servers, bounds)
@@ -46,14 +47,14 @@ def test_c1_resnet20_constant_full_vector_full_log():
 def test_c2_adaptive_full_log_sampled():
     wl = synth.workload("c2_adaptive_1p7m")
     w0, pool, ev = wl.w0(), U.host_pool(wl), wl.log()
-    sampled_check(wl, w0, pool, U.to_device(pool), ev, (32, 8, 1))
+    sampled_check(wl, w0, pool, U.to_device(pool), ev, (32, 8, 256, 1280, 1))
 
 
 def test_c3_resnet50_adaptive_as_benchmarked():
     wl = synth.workload("c3_resnet50_adaptive")
     w0, pool, ev = wl.w0(), U.host_pool(wl), wl.log()
     dpool = U.to_device(pool)
-    sampled_check(wl, w0, pool, dpool, ev, (32, 8, 1))
+    sampled_check(wl, w0, pool, dpool, ev, (32, 8, 256, 1))
     # full vector on the first 64 pushes
     prefix = ev[: wl.M + 2 * 64]
     servers, bounds = U.cpu_replay_ranges(wl, prefix, w0, pool, os.cpu_count() or 1)
@@ -67,4 +68,4 @@ def test_c4_vgg16_bf16_full_log_sampled(name):
     wl = synth.workload(name)
     w0, pool, ev = wl.w0(), U.host_pool(wl), wl.log()
     assert pool.dtype == np.uint16
-    sampled_check(wl, w0, pool, U.to_device(pool), ev, (32, 1))
+    sampled_check(wl, w0, pool, U.to_device(pool), ev, (32, 8, 1))
